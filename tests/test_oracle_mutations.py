@@ -1,0 +1,69 @@
+"""Plants single mistakes in a copy of the CPU checker and verifies that the pin
+suite (tests/test_oracle_pins.py) rejects every one of them.  Everything here runs
+on the CPU; the planted copies are compiled into a temporary directory."""
+import os
+import subprocess
+import sys
+from concurrent.futures import ThreadPoolExecutor
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "mqg_oracle.c")
+
+# (name, text in the source, replacement)
+MUTANTS = [
+    ("dropped_half_L", "float t = fmaf(x[i], inv, halfL);", "float t = fmaf(x[i], inv, 0.0f);"),
+    ("unfused_encode", "float t = fmaf(x[i], inv, halfL);", "float t = x[i] * inv + halfL;"),
+    ("wrong_sign_x", "float t = fmaf(x[i], inv, halfL);", "float t = fmaf(-x[i], inv, halfL);"),
+    ("scale_not_doubled", "float two_s = 2.0f * s;", "float two_s = s;"),
+    ("uncentred_draw", "((float)h[i] + 0.5f) * (1.0f / 65536.0f)", "((float)h[i]) * (1.0f / 65536.0f)"),
+    ("round_down_always", "(u < r) ? 1 : 0", "0"),
+    ("inverted_compare", "(u < r) ? 1 : 0", "(u > r) ? 1 : 0"),
+    ("pack_msb_first", "if ((q[i] >> j) & 1u) {", "if ((q[i] >> (bits - 1 - j)) & 1u) {"),
+    ("pack_word_bit_reversed", "words[pos >> 5] |= (uint32_t)1u << (pos & 31u);",
+     "words[pos >> 5] |= (uint32_t)0x80000000u >> (pos & 31u);"),
+    ("levels_2_pow_k", "const int L = (1 << bits) - 1;", "const int L = (1 << bits);"),
+    ("dequant_missing_factor_2", "(float)(2 * (int)q[i] - L)", "(float)((int)q[i] - L)"),
+    ("dequant_double_rounding", "xhat[i] = level * hstep;", "xhat[i] = (level * s) / Lf;"),
+    ("apply_unfused", "params[i] = fmaf(-lr, acc[i], params[i]);", "params[i] = params[i] - lr * acc[i];"),
+    ("apply_wrong_sign", "params[i] = fmaf(-lr, acc[i], params[i]);", "params[i] = fmaf(lr, acc[i], params[i]);"),
+    ("philox_constants_swapped", "(uint64_t)0xD2511F53u * (uint64_t)c0", "(uint64_t)0xCD9E8D57u * (uint64_t)c0"),
+    ("philox_nine_rounds", "round < 10", "round < 9"),
+    ("philox_key_not_bumped", "k1 += 0xBB67AE85u;", ""),
+    ("draw_wrong_half", "(16u * (e & 1u))", "(16u * ((e & 1u) ^ 1u))"),
+    ("draw_worker_step_swapped", "(uint32_t)(blk >> 32), worker, step }", "(uint32_t)(blk >> 32), step, worker }"),
+    ("scale_signed_max", "float a = fabsf(x[i]);", "float a = x[i];"),
+    ("flush_threshold", "ldexpf(1.0f, -96)", "ldexpf(1.0f, -90)"),
+    ("bf16_low_half", "(uint32_t)in[i] << 16", "(uint32_t)in[i]"),
+    ("sum_skips_last_worker", "for (int w = 0; w < W; ++w) {\n        mqo_unpack", "for (int w = 0; w < W - (W > 2); ++w) {\n        mqo_unpack"),
+    ("zero_bucket_minus_zero", "if (s == 0.0f) { xhat[i] = 0.0f; continue; }", "if (s == 0.0f) { xhat[i] = -0.0f; continue; }"),
+]
+
+
+def _run(args):
+    name, old, new, tmpdir = args
+    text = open(SRC).read()
+    assert text.count(old) >= 1, name
+    mutated = text.replace(old, new, 1)
+    c = os.path.join(tmpdir, name + ".c")
+    so = os.path.join(tmpdir, name + ".so")
+    with open(c, "w") as f:
+        f.write(mutated)
+    subprocess.run(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math", "-fPIC",
+                    "-shared", "-o", so, c, "-lm"], check=True)
+    env = dict(os.environ, MQG_ORACLE_LIB=so)
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+                        os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+                       cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
+    return name, r.returncode, r.stdout[-400:]
+
+
+def test_every_planted_mistake_is_caught(tmp_path):
+    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS]
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 2)) as ex:
+        results = list(ex.map(_run, jobs))
+    survivors = [name for name, rc, _ in results if rc == 0]
+    assert not survivors, "pins do not catch: %s" % survivors
+    crashed = [(name, out) for name, rc, out in results if rc not in (0, 1)]
+    assert not crashed, crashed
