@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the MQGrad hot path on B200: quantize+pack and unpack+accumulate+update.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload (the configuration the headline metric is quoted on): one flat gradient of
+n = 25,000,000 fp32 per worker, W = 8 simulated workers, iid Laplace(0, 1e-4), bucket 2048,
+bit widths 1..8.  One step = one pass of the whole path for every bit width: 8 x W quantize
+launches (each reads a distinct 100 MB gradient) followed by 8 fused server launches (each
+reads W code buffers and updates its own 100 MB parameter replica), so every launch reads
+inputs that have been evicted from L2 (> 1.7 GB cycles between reuses).
+
+Prints ONE JSON line (rank 0).  `value` is GB/s of fp32 gradient through the whole path
+(8 * W * 4n bytes per step / step time) with all inputs resident in HBM; `e2e` is the same
+metric with the gradients starting in pinned host memory and the updated parameters read
+back, copies inside the timed region; `roofline` describes the dominant kernel
+(quantize_pack_kernel); `per_bits` lists both kernels for every bit width; `cpu_baseline` is
+the scalar CPU checker timed on a bounded sample of the same workload.
+
+--impl reference times the CPU checker alone (rank 0 only).
+With --gpus N > 1 (under torchrun) every rank runs an independent replica of the workload
+on its own GPU; there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+N_ELEMS = 25_000_000
+N_WORKERS = 8
+BUCKET = 2048
+ALL_BITS = list(range(1, 9))
+LAPLACE_SCALE = 1e-4
+LR = 0.1 / N_WORKERS
+PHILOX_SEED = 2
+METRIC = "quantize+pack and dequant+accumulate+update GB/s (fp32 grad) per bit width; % HBM peak"
+UNIT = "GB/s of fp32 gradient through quantize+pack -> unpack+accumulate+update"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def quantize_bytes(n, bits, bucket):
+    """Algorithmic bytes of one quantize launch: read fp32, write codes and scales."""
+    return 4 * n + 4 * ((n * bits + 31) // 32) + 4 * ((n + bucket - 1) // bucket)
+
+
+def server_bytes(n, bits, bucket, W):
+    """Algorithmic bytes of one fused server launch: W code streams + W scale arrays + params r/w."""
+    return W * (4 * ((n * bits + 31) // 32) + 4 * ((n + bucket - 1) // bucket)) + 8 * n
+
+
+# --------------------------------------------------------------------------------------
+# clocks: sampled with NVML while the timed region runs (read-only queries)
+# --------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+        0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+        0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = device_index
+            if visible:
+                ids = [v for v in visible.split(",") if v.strip() != ""]
+                if device_index < len(ids) and ids[device_index].strip().isdigit():
+                    phys = int(ids[device_index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------
+# CPU checker leg (the oracle as it stands; bench.py is one of the few places allowed to run it)
+# --------------------------------------------------------------------------------------
+def oracle_pass(grads, n_s, bits_list, threads):
+    """One pass of the whole path on the first n_s elements of every worker, on the CPU checker.
+    Bit widths are independent and run on `threads` host threads.  Returns seconds."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    from oracle import mqg_oracle as O
+
+    def one(bits):
+        codes, scales = [], []
+        for w, g in enumerate(grads):
+            c, s = O.quantize(g[:n_s], bits, BUCKET, PHILOX_SEED, worker=w)
+            codes.append(c), scales.append(s)
+        p = np.zeros(n_s, np.float32)
+        O.server_step(codes, scales, bits, n_s, BUCKET, p, LR)
+        return float(p[0])
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(one, bits_list))
+    return time.perf_counter() - t0
+
+
+def host_threads():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def make_grads(n, workers):
+    from concurrent.futures import ThreadPoolExecutor
+
+    from paper_1804_08066_b200 import workloads as wl
+    with ThreadPoolExecutor(max_workers=min(workers, host_threads())) as ex:
+        return list(ex.map(lambda w: wl.laplace(n, LAPLACE_SCALE, config=2, worker=w), range(workers)))
+
+
+def cpu_baseline(grads, target_seconds=20.0):
+    cores = host_threads()
+    threads = max(1, min(cores, len(ALL_BITS)))
+    probe = 32 * BUCKET
+    t = oracle_pass(grads, probe, ALL_BITS, threads)
+    per_elem = t / probe
+    n_s = int(target_seconds / threads / max(per_elem, 1e-12))     # ~target_seconds of CPU work
+    n_s = max(BUCKET, min(N_ELEMS // BUCKET * BUCKET, n_s // BUCKET * BUCKET))
+    secs = oracle_pass(grads, n_s, ALL_BITS, threads)
+    gbs = len(ALL_BITS) * len(grads) * 4 * n_s / secs / 1e9
+    return {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "first %d of %d elements of each of %d workers, bits 1..8, one pass in %.2f s"
+                      % (n_s, N_ELEMS, len(grads), secs)}, n_s
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    t_budget = 150.0
+    n_probe = 16 * BUCKET
+    grads = make_grads(max(n_probe, 2_000_000), N_WORKERS)
+    cores = host_threads()
+    threads = max(1, min(cores, len(ALL_BITS)))
+    t = oracle_pass(grads, n_probe, ALL_BITS, threads)
+    per_elem = t / n_probe
+    total_steps = args.steps + args.warmup
+    n_s = int(t_budget / max(total_steps, 1) / max(per_elem, 1e-12))
+    n_s = max(BUCKET, min(grads[0].size // BUCKET * BUCKET, n_s // BUCKET * BUCKET))
+    for _ in range(args.warmup):
+        oracle_pass(grads, n_s, ALL_BITS, threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(grads, n_s, ALL_BITS, threads)
+    dt = time.perf_counter() - t0
+    gbs = args.steps * len(ALL_BITS) * N_WORKERS * 4 * n_s / dt / 1e9
+    sample = ("each step = first %d of %d elements of each of %d workers, bits 1..8"
+              % (n_s, N_ELEMS, N_WORKERS))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": workload_config(),
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config():
+    return {"workload": "configs[1]: flat ResNet-50-sized gradient, n=25,000,000 fp32 per worker, W=8, "
+                        "iid Laplace(0,1e-4), bucket 2048, bits 1..8",
+            "n": N_ELEMS, "workers": N_WORKERS, "bucket": BUCKET, "bits": ALL_BITS,
+            "l2": "inputs larger than L2: every launch reads buffers last touched > 1.7 GB of traffic ago",
+            "multi_gpu": "replicas only"}
+
+
+# --------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+
+    import paper_1804_08066_b200 as mqg
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libmqgrad has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    n, W, B = N_ELEMS, N_WORKERS, BUCKET
+    lib = mqg.raw_library()
+    host_grads = make_grads(n, W)
+    pinned = [torch.from_numpy(g).pin_memory() for g in host_grads]
+    grads = [p.cuda(non_blocking=True) for p in pinned]
+    from paper_1804_08066_b200 import workloads as wl
+    params0 = torch.from_numpy(wl.params(n, 0.05, config=2)).cuda()
+    params = {b: params0.clone() for b in ALL_BITS}
+    codes = {b: [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(W)]
+             for b in ALL_BITS}
+    scales = {b: [torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(W)]
+              for b in ALL_BITS}
+    host_params = torch.empty(n, dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    sptr = C.c_void_p(stream.cuda_stream)
+    code_tab = {b: (C.c_void_p * W)(*[t.data_ptr() for t in codes[b]]) for b in ALL_BITS}
+    scale_tab = {b: (C.c_void_p * W)(*[t.data_ptr() for t in scales[b]]) for b in ALL_BITS}
+
+    def check(rc):
+        if rc != 0:
+            raise RuntimeError("libmqgrad: %d %s" % (rc, mqg.mqg_last_error()))
+
+    def quantize_all(b, step_no):
+        for w in range(W):
+            check(lib.mqg_quantize(grads[w].data_ptr(), n, b, B, PHILOX_SEED, codes[b][w].data_ptr(),
+                                   scales[b][w].data_ptr(), 0, w, step_no, 0, sptr))
+
+    def server(b):
+        check(lib.mqg_server_step(code_tab[b], scale_tab[b], W, b, n, B, params[b].data_ptr(), LR,
+                                  None, sptr))
+
+    def step(step_no, events=None):
+        for b in ALL_BITS:
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            quantize_all(b, step_no)
+            if events is not None:
+                e1.record(stream)
+                events.append(("q", b, e0, e1))
+        for b in ALL_BITS:
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            server(b)
+            if events is not None:
+                e1.record(stream)
+                events.append(("s", b, e0, e1))
+
+    def e2e_step(step_no):
+        for b in ALL_BITS:
+            for w in range(W):
+                grads[w].copy_(pinned[w], non_blocking=True)
+                check(lib.mqg_quantize(grads[w].data_ptr(), n, b, B, PHILOX_SEED, codes[b][w].data_ptr(),
+                                       scales[b][w].data_ptr(), 0, w, step_no, 0, sptr))
+            server(b)
+            host_params.copy_(params[b], non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    events = []
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_begin.record(stream)
+        for i in range(args.steps):
+            step(args.warmup + i, events)
+        t_end.record(stream)
+        barrier()
+    total_ms = max_over_ranks(t_begin.elapsed_time(t_end))
+    ms_per_step = total_ms / args.steps
+    grad_bytes_per_step = len(ALL_BITS) * W * 4 * n
+    value = world * grad_bytes_per_step / (ms_per_step * 1e-3) / 1e9
+
+    q_ms = {b: [] for b in ALL_BITS}
+    s_ms = {b: [] for b in ALL_BITS}
+    for kind, b, e0, e1 in events:
+        (q_ms if kind == "q" else s_ms)[b].append(e0.elapsed_time(e1))
+    peak, peak_kind = measured_hbm_peak()
+    per_bits = []
+    q_bytes_total = q_time_total = 0.0
+    s_bytes_total = s_time_total = 0.0
+    for b in ALL_BITS:
+        tq = float(np.mean(q_ms[b])) / W * 1e-3            # per quantize launch
+        ts = float(np.mean(s_ms[b])) * 1e-3
+        qb, sb = quantize_bytes(n, b, B), server_bytes(n, b, B, W)
+        q_bytes_total += qb * W; q_time_total += tq * W
+        s_bytes_total += sb; s_time_total += ts
+        per_bits.append({
+            "bits": b,
+            "quantize_us": tq * 1e6, "quantize_grad_gbs": 4 * n / tq / 1e9, "quantize_moved_gbs": qb / tq / 1e9,
+            "quantize_frac_of_measured": qb / tq / 1e9 / peak, "quantize_frac_of_8tbs": qb / tq / 1e9 / NOMINAL_HBM_GBS,
+            "server_us": ts * 1e6, "server_grad_gbs": 4 * n * W / ts / 1e9, "server_moved_gbs": sb / ts / 1e9,
+            "server_frac_of_measured": sb / ts / 1e9 / peak, "server_frac_of_8tbs": sb / ts / 1e9 / NOMINAL_HBM_GBS,
+            "wire_bytes_per_worker": mqg.mqg_wire_bytes(n, b, B),
+        })
+    q_achieved = q_bytes_total / q_time_total / 1e9
+    s_achieved = s_bytes_total / s_time_total / 1e9
+    roofline = {"kernel": "quantize_pack_kernel (all bit widths, %d launches per step)" % (len(ALL_BITS) * W),
+                "bound": "hbm", "achieved": q_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
+                "unit": "GB/s", "frac": q_achieved / peak, "traffic": None,
+                "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
+    roofline_server = {"kernel": "server_kernel (fused, all bit widths, %d launches per step)" % len(ALL_BITS),
+                       "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
+                       "unit": "GB/s", "frac": s_achieved / peak, "traffic": None}
+
+    # ---- end to end from pinned host buffers
+    e2e_steps = max(1, min(args.steps, 3))
+    e2e_step(0)
+    barrier()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(1 + i)
+    b1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(b0.elapsed_time(b1)) / e2e_steps
+    e2e = {"value": world * grad_bytes_per_step / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+           "h2d_bytes_per_step": grad_bytes_per_step, "d2h_bytes_per_step": len(ALL_BITS) * 4 * n,
+           "ms_per_step": e2e_ms, "steps": e2e_steps}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu, _ = cpu_baseline(host_grads)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(), "clocks": clocks.summary(), "e2e": e2e,
+            "gpu_launches": args.steps * len(ALL_BITS) * (W + 1),
+            "roofline": roofline, "roofline_server": roofline_server, "per_bits": per_bits,
+        }
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

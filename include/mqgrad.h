@@ -1,0 +1,146 @@
+/*
+ * mqgrad.h -- C ABI of libmqgrad: the per-iteration gradient codec of MQGrad
+ * (arXiv 1804.08066) for one NVIDIA B200 (sm_100a).
+ *
+ * The paper's data path per training iteration (Algorithm 1, Section 3.2):
+ *   worker:  g~ <- Quantize(g, K)                         (WorkerIterate)
+ *   server:  g_p <- De-quantize(g~_p) for p = 1..P,
+ *            g <- sum_p g_p / P,  w <- w - eta * g        (ReceiveQGThenSendQG, steps 6-7 of Fig. 3)
+ * The paper leaves the codec itself to an external page; this library fixes it as:
+ * a symmetric K-bit affine grid on [-s, +s] per bucket (s = max |x| of the bucket),
+ * unbiased stochastic rounding with 16 random bits per element from Philox4x32-10,
+ * and LSB-first packing of the K-bit codes into little-endian 32-bit words.
+ *
+ * Conventions that hold for every call
+ *   - Every data pointer is caller-owned DEVICE memory unless stated otherwise; the
+ *     library never allocates, frees or keeps device memory.  Arrays of pointers
+ *     (codes[W], scales[W]) and segment tables are HOST arrays, read during the call.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and return without waiting for it.
+ *   - Return value: MQG_OK, or a negative mqg_status; nothing is thrown and nothing
+ *     aborts.  Arguments are checked on the host before any launch; on an error
+ *     nothing has been enqueued.  mqg_last_error() gives the calling thread's message.
+ *   - n == 0 is a valid no-op.  Inputs must be finite; results for NaN/Inf are unspecified.
+ *   - Output buffers must not overlap inputs, except `params`, updated in place.
+ *   - grad, params, acc and codes must be 16-byte aligned; scales 4-byte aligned.
+ *   - 1 <= bits <= 8.  L = 2^bits - 1.
+ *   - bucket >= 1, and bucket % 32 == 0 unless bucket >= n (one bucket), so that every
+ *     bucket's codes start on a word boundary for every bit width.
+ */
+#ifndef MQGRAD_H_
+#define MQGRAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int mqg_status;
+enum {
+    MQG_OK = 0,
+    MQG_ERR_INVALID = -1,          /* null pointer, bad bucket, bad segment table, overlapping sizes */
+    MQG_ERR_BITS = -2,             /* bits outside 1..8 */
+    MQG_ERR_ALIGN = -3,            /* a buffer is not aligned as required */
+    MQG_ERR_TOO_MANY_WORKERS = -4, /* W outside 1..MQG_MAX_WORKERS */
+    MQG_ERR_CUDA = -5              /* a CUDA runtime call failed; see mqg_last_error() */
+};
+
+typedef enum { MQG_F32 = 0, MQG_BF16 = 1 } mqg_dtype;
+
+#define MQG_MAX_WORKERS 32
+
+/* Number of 32-bit words of one worker's packed stream: ceil(n * bits / 32).  Host-only helper. */
+size_t mqg_code_words(uint64_t n, int bits);
+
+/* Number of buckets (= scales) for n elements: ceil(n / bucket).  Host-only helper. */
+size_t mqg_num_buckets(uint64_t n, uint64_t bucket);
+
+/* Bytes one worker sends for n elements: 4 * code_words + 4 * num_buckets (reported, never timed). */
+size_t mqg_wire_bytes(uint64_t n, int bits, uint64_t bucket);
+
+/*
+ * Quantize(g, K) of Algorithm 1 (WorkerIterate), fused with packing.
+ *   grad        [in]  n elements of `dtype` (fp32, or bf16 widened exactly to fp32 in the kernel)
+ *   codes       [out] mqg_code_words(n, bits) words; code i at bits [i*bits, i*bits+bits) of the
+ *                     stream, bit j of the stream = bit (j % 32) of word j / 32; pad bits are zero
+ *   scales      [out] mqg_num_buckets(n, bucket) floats; s_k = max |x| of bucket k, flushed to 0
+ *                     below 2^-96 (then every code of the bucket is 0)
+ *   seed, worker, step, elem_offset
+ *                     key the random draws: element i draws from Philox4x32-10 with key = seed and
+ *                     counter = ((elem_offset + i) / 8, worker, step), 16 bits per element, so the
+ *                     codes are a pure function of the arguments (reproducible, order-free).
+ *                     elem_offset is the element's position in the flat model; multiples of 8
+ *                     take the fast path.
+ * Per element: t = fma(x, L / (2 s), L / 2) in fp32, code = floor(t) + [u < t - floor(t)],
+ * u = (h + 1/2) / 65536.
+ */
+mqg_status mqg_quantize(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                        uint32_t* codes, float* scales,
+                        mqg_dtype dtype, uint32_t worker, uint32_t step, uint64_t elem_offset,
+                        void* cuda_stream);
+
+/*
+ * De-quantize + sum of Algorithm 1 (ReceiveQGThenSendQG, before the division by P):
+ *   acc[i] = ((x^_0[i] + x^_1[i]) + ... ) in worker order 0..W-1, fp32,
+ *   x^_w[i] = (2 q - L) * (s / L) with one rounding for s / L and one for the product;
+ *   a zero-scale bucket decodes to +0.
+ *   codes, scales  [in]  HOST arrays of W device pointers, laid out as mqg_quantize writes them
+ *   acc            [out] n floats; overwritten, or (add_into_acc != 0) the sum continues from the
+ *                        value already there: acc = ((acc + x^_0) + x^_1) + ...
+ */
+mqg_status mqg_dequant_accumulate(const uint32_t* const* codes, const float* const* scales, int W,
+                                  int bits, uint64_t n, float* acc,
+                                  uint64_t bucket, int add_into_acc, void* cuda_stream);
+
+/*
+ * w <- w - eta * g of Algorithm 1 (WorkerIterate's update), one fused multiply-add per element:
+ * params[i] = fma(-lr, acc[i], params[i]).  Pass lr = eta / P to apply the mean of P workers.
+ */
+mqg_status mqg_apply(float* params, const float* acc, float lr, uint64_t n, void* cuda_stream);
+
+/*
+ * The server's whole step in one pass over memory (steps 6-7 of Fig. 3, Section 3.2): unpack,
+ * de-quantize and sum W workers' buffers and update the shared parameters, with exactly the
+ * roundings of mqg_dequant_accumulate followed by mqg_apply.
+ *   params   [in/out] n floats, updated in place
+ *   acc_out  [out]    optional (may be NULL): the summed gradient, n floats
+ */
+mqg_status mqg_server_step(const uint32_t* const* codes, const float* const* scales, int W, int bits,
+                           uint64_t n, uint64_t bucket, float* params, float lr, float* acc_out,
+                           void* cuda_stream);
+
+/*
+ * Per-layer scale ("gradient quantization is applied to these two layers", Section 4.1): the flat
+ * gradient is cut into nseg segments; segment j = elements [seg_off[j], seg_off[j+1]) is ONE bucket
+ * with scale scales[j], and its bit stream starts on a word boundary at word code_off[j].
+ *   seg_off   [in] HOST array of nseg+1 non-decreasing element offsets (seg_off[0] may be > 0)
+ *   code_off  [in] HOST array of nseg+1 word offsets; code_off[j+1] - code_off[j] >=
+ *                  mqg_code_words(seg_off[j+1] - seg_off[j], bits)
+ *   grad      [in] the whole flat gradient (element 0 of the array is flat index 0)
+ *   codes     [out] code_off[nseg] words;  scales [out] nseg floats
+ * Element i of segment j draws with position elem_offset + seg_off[j] + i.  Empty segments get
+ * scale 0.  The gradient is read twice (max pass, encode pass).
+ */
+mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg_off,
+                                 const uint64_t* code_off, int bits, uint64_t seed,
+                                 uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                                 uint32_t step, uint64_t elem_offset, void* cuda_stream);
+
+/* mqg_server_step for buffers written by mqg_quantize_segments (same segment tables). */
+mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* const* scales, int W,
+                                    int bits, int nseg, const uint64_t* seg_off,
+                                    const uint64_t* code_off, float* params, float lr,
+                                    float* acc_out, void* cuda_stream);
+
+/* Message of the last error returned to the calling thread ("" if none).  Never NULL. */
+const char* mqg_last_error(void);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int mqg_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MQGRAD_H_ */

@@ -1,0 +1,175 @@
+"""libmqgrad for B200: Python binding of the C ABI in include/mqgrad.h.
+
+The binding only marshals arguments: torch CUDA tensors supply the device pointers and the
+current torch stream supplies the CUDA stream; every step of the path runs in the CUDA
+kernels of libmqgrad.so.  There is no CPU fallback: a missing library or a CPU tensor
+raises.
+
+Function names and argument order follow the C ABI:
+  mqg_quantize, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
+  mqg_quantize_segments, mqg_server_step_segments, mqg_code_words, mqg_num_buckets,
+  mqg_wire_bytes, mqg_last_error, mqg_version.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmqgrad.so")
+
+MQG_OK = 0
+MQG_ERR_INVALID = -1
+MQG_ERR_BITS = -2
+MQG_ERR_ALIGN = -3
+MQG_ERR_TOO_MANY_WORKERS = -4
+MQG_ERR_CUDA = -5
+MQG_F32, MQG_BF16 = 0, 1
+MQG_MAX_WORKERS = 32
+
+
+class MqgError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("libmqgrad status %d: %s" % (status, message))
+        self.status = status
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libmqgrad.so is not built (%s); run `python -m paper_1804_08066_b200.build`. "
+            "There is no fallback path." % LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
+    u64, u32, i32, vp, f32 = C.c_uint64, C.c_uint32, C.c_int, C.c_void_p, C.c_float
+    sigs = {
+        "mqg_code_words": (C.c_size_t, [u64, i32]),
+        "mqg_num_buckets": (C.c_size_t, [u64, u64]),
+        "mqg_wire_bytes": (C.c_size_t, [u64, i32, u64]),
+        "mqg_last_error": (C.c_char_p, []),
+        "mqg_version": (i32, []),
+        "mqg_quantize": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
+        "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
+        "mqg_apply": (i32, [vp, vp, f32, u64, vp]),
+        "mqg_server_step": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
+        "mqg_quantize_segments": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
+        "mqg_server_step_segments": (i32, [vp, vp, i32, i32, i32, vp, vp, vp, f32, vp, vp]),
+    }
+    for name, (res, args) in sigs.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+_lib = _load()
+
+
+def _check(status: int) -> None:
+    if status != MQG_OK:
+        raise MqgError(status, _lib.mqg_last_error().decode())
+
+
+def _dev_ptr(t, what: str) -> int:
+    import torch
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor (libmqgrad has no CPU path)" % what)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % what)
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr_table(tensors, what: str):
+    return (C.c_void_p * len(tensors))(*[_dev_ptr(t, "%s[%d]" % (what, i))
+                                         for i, t in enumerate(tensors)])
+
+
+def _u64_table(values):
+    vals = [int(v) for v in values]
+    return (C.c_uint64 * len(vals))(*vals)
+
+
+def mqg_code_words(n: int, bits: int) -> int:
+    return int(_lib.mqg_code_words(n, bits))
+
+
+def mqg_num_buckets(n: int, bucket: int) -> int:
+    return int(_lib.mqg_num_buckets(n, bucket))
+
+
+def mqg_wire_bytes(n: int, bits: int, bucket: int) -> int:
+    return int(_lib.mqg_wire_bytes(n, bits, bucket))
+
+
+def mqg_last_error() -> str:
+    return _lib.mqg_last_error().decode()
+
+
+def mqg_version() -> int:
+    return int(_lib.mqg_version())
+
+
+def _grad_dtype(grad) -> int:
+    import torch
+    if grad.dtype == torch.float32:
+        return MQG_F32
+    if grad.dtype == torch.bfloat16:
+        return MQG_BF16
+    raise TypeError("grad must be float32 or bfloat16, got %s" % grad.dtype)
+
+
+def mqg_quantize(grad, n: int, bits: int, bucket: int, seed: int, codes, scales,
+                 worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    """Quantize(g, K): writes `codes` (uint32/int32 words) and `scales` (float32)."""
+    _check(_lib.mqg_quantize(_dev_ptr(grad, "grad") if n else None, n, bits, bucket,
+                             seed & 0xFFFFFFFFFFFFFFFF,
+                             _dev_ptr(codes, "codes") if n else None,
+                             _dev_ptr(scales, "scales") if n else None,
+                             _grad_dtype(grad), worker, step, elem_offset, _stream()))
+
+
+def mqg_dequant_accumulate(codes, scales, W: int, bits: int, n: int, acc, bucket: int,
+                           add_into_acc: bool = False) -> None:
+    _check(_lib.mqg_dequant_accumulate(_ptr_table(codes, "codes"), _ptr_table(scales, "scales"),
+                                       W, bits, n, _dev_ptr(acc, "acc") if n else None, bucket,
+                                       1 if add_into_acc else 0, _stream()))
+
+
+def mqg_apply(params, acc, lr: float, n: int) -> None:
+    _check(_lib.mqg_apply(_dev_ptr(params, "params") if n else None,
+                          _dev_ptr(acc, "acc") if n else None, lr, n, _stream()))
+
+
+def mqg_server_step(codes, scales, W: int, bits: int, n: int, bucket: int, params, lr: float,
+                    acc_out=None) -> None:
+    _check(_lib.mqg_server_step(_ptr_table(codes, "codes"), _ptr_table(scales, "scales"), W, bits,
+                                n, bucket, _dev_ptr(params, "params") if n else None, lr,
+                                _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
+                                _stream()))
+
+
+def mqg_quantize_segments(grad, seg_off, code_off, bits: int, seed: int, codes, scales,
+                          worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    nseg = len(seg_off) - 1
+    _check(_lib.mqg_quantize_segments(_dev_ptr(grad, "grad"), nseg, _u64_table(seg_off),
+                                      _u64_table(code_off), bits, seed & 0xFFFFFFFFFFFFFFFF,
+                                      _dev_ptr(codes, "codes"), _dev_ptr(scales, "scales"),
+                                      _grad_dtype(grad), worker, step, elem_offset, _stream()))
+
+
+def mqg_server_step_segments(codes, scales, W: int, bits: int, seg_off, code_off, params,
+                             lr: float, acc_out=None) -> None:
+    nseg = len(seg_off) - 1
+    _check(_lib.mqg_server_step_segments(_ptr_table(codes, "codes"), _ptr_table(scales, "scales"),
+                                         W, bits, nseg, _u64_table(seg_off), _u64_table(code_off),
+                                         _dev_ptr(params, "params"), lr,
+                                         _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
+                                         _stream()))
+
+
+def raw_library() -> C.CDLL:
+    """The ctypes handle, for callers that pass raw device pointers themselves."""
+    return _lib

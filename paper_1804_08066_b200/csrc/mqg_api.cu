@@ -1,0 +1,249 @@
+// C ABI of libmqgrad: argument checks, dispatch to the kernel launchers, error reporting.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/mqgrad.h"
+#include "mqg_common.cuh"
+#include "mqg_internal.h"
+
+namespace {
+
+thread_local char g_err[256] = "";
+
+mqg_status fail(mqg_status code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+mqg_status cuda_fail(const char* what, cudaError_t err)
+{
+    return fail(MQG_ERR_CUDA, "%s: %s", what, cudaGetErrorString(err));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+mqg_status check_bits(int bits)
+{
+    if (bits < 1 || bits > 8) return fail(MQG_ERR_BITS, "bits = %d is outside 1..8", bits);
+    return MQG_OK;
+}
+
+mqg_status check_bucket(uint64_t n, uint64_t bucket)
+{
+    if (bucket == 0) return fail(MQG_ERR_INVALID, "bucket must be >= 1");
+    if (bucket < n && bucket % 32 != 0)
+        return fail(MQG_ERR_INVALID, "bucket = %llu must be a multiple of 32 (or >= n)",
+                    (unsigned long long)bucket);
+    return MQG_OK;
+}
+
+// With `empty` (nothing to process) only W is checked: the buffers may be null.
+mqg_status check_workers(const uint32_t* const* codes, const float* const* scales, int W,
+                         bool empty, mqg::WorkerPtrs* out)
+{
+    if (W < 1 || W > MQG_MAX_WORKERS)
+        return fail(MQG_ERR_TOO_MANY_WORKERS, "W = %d is outside 1..%d", W, MQG_MAX_WORKERS);
+    if (empty) return MQG_OK;
+    if (!codes || !scales) return fail(MQG_ERR_INVALID, "codes / scales pointer table is null");
+    for (int w = 0; w < W; ++w) {
+        if (!codes[w] || !scales[w])
+            return fail(MQG_ERR_INVALID, "worker %d: codes or scales buffer is null", w);
+        if (!aligned16(codes[w])) return fail(MQG_ERR_ALIGN, "worker %d: codes not 16-byte aligned", w);
+        if (!aligned4(scales[w])) return fail(MQG_ERR_ALIGN, "worker %d: scales not 4-byte aligned", w);
+        out->codes[w] = codes[w];
+        out->scales[w] = scales[w];
+    }
+    for (int w = W; w < mqg::kMaxWorkers; ++w) { out->codes[w] = nullptr; out->scales[w] = nullptr; }
+    return MQG_OK;
+}
+
+// Validates a segment table and cuts it into chunks of at most kMaxSegmentsPerLaunch segments;
+// calls fn(table, first_segment_index) for each chunk that has at least one tile.
+template <typename Fn>
+mqg_status for_each_chunk(int nseg, const uint64_t* seg_off, const uint64_t* code_off, int bits,
+                          Fn&& fn)
+{
+    if (nseg < 0) return fail(MQG_ERR_INVALID, "nseg = %d is negative", nseg);
+    if (nseg == 0) return MQG_OK;
+    if (!seg_off || !code_off) return fail(MQG_ERR_INVALID, "segment table is null");
+    for (int j = 0; j < nseg; ++j) {
+        if (seg_off[j + 1] < seg_off[j]) return fail(MQG_ERR_INVALID, "seg_off decreases at %d", j);
+        const uint64_t len = seg_off[j + 1] - seg_off[j];
+        const uint64_t need = (len * (uint64_t)bits + 31) / 32;
+        if (code_off[j + 1] < code_off[j] || code_off[j + 1] - code_off[j] < need)
+            return fail(MQG_ERR_INVALID, "code_off leaves segment %d fewer than %llu words", j,
+                        (unsigned long long)need);
+    }
+    const uint64_t tile_elems = (uint64_t)mqg::kMaxTileRows * 32;
+    int j = 0;
+    while (j < nseg) {
+        mqg::SegmentTable tab;
+        std::memset(&tab, 0, sizeof(tab));
+        int k = 0;
+        uint64_t tiles = 0;
+        while (j + k < nseg && k < mqg::kMaxSegmentsPerLaunch) {
+            const uint64_t len = seg_off[j + k + 1] - seg_off[j + k];
+            const uint64_t t = (len + tile_elems - 1) / tile_elems;
+            if (tiles + t > 0x7FFFFFFFull) break;
+            tab.tile_start[k] = (uint32_t)tiles;
+            tab.seg_off[k] = seg_off[j + k];
+            tab.code_off[k] = code_off[j + k];
+            tiles += t;
+            ++k;
+        }
+        if (k == 0) return fail(MQG_ERR_INVALID, "segment %d is too large for one launch", j);
+        tab.tile_start[k] = (uint32_t)tiles;
+        tab.seg_off[k] = seg_off[j + k];
+        tab.nseg = k;
+        const mqg_status st = fn(tab, j);
+        if (st != MQG_OK) return st;
+        j += k;
+    }
+    return MQG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mqg_code_words(uint64_t n, int bits) { return (size_t)((n * (uint64_t)bits + 31) / 32); }
+
+size_t mqg_num_buckets(uint64_t n, uint64_t bucket)
+{
+    return bucket ? (size_t)((n + bucket - 1) / bucket) : 0;
+}
+
+size_t mqg_wire_bytes(uint64_t n, int bits, uint64_t bucket)
+{
+    return 4 * mqg_code_words(n, bits) + 4 * mqg_num_buckets(n, bucket);
+}
+
+const char* mqg_last_error(void) { return g_err; }
+
+int mqg_version(void) { return 100; }
+
+mqg_status mqg_quantize(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                        uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                        uint32_t step, uint64_t elem_offset, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (n == 0) return MQG_OK;
+    if (!grad || !codes || !scales) return fail(MQG_ERR_INVALID, "grad, codes or scales is null");
+    if (!aligned16(grad)) return fail(MQG_ERR_ALIGN, "grad not 16-byte aligned");
+    if (!aligned16(codes)) return fail(MQG_ERR_ALIGN, "codes not 16-byte aligned");
+    if (!aligned4(scales)) return fail(MQG_ERR_ALIGN, "scales not 4-byte aligned");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t eff = bucket < n ? bucket : n;
+    cudaError_t err;
+    if (eff <= (uint64_t)mqg::kMaxFusedBucket)
+        err = mqg::launch_quantize_fused(grad, n, bits, bucket, seed, codes, scales, (int)dtype,
+                                         worker, step, elem_offset, stream);
+    else
+        err = mqg::launch_quantize_big_buckets(grad, n, bits, bucket, seed, codes, scales, (int)dtype,
+                                               worker, step, elem_offset, stream);
+    if (err != cudaSuccess) return cuda_fail("mqg_quantize", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_dequant_accumulate(const uint32_t* const* codes, const float* const* scales, int W,
+                                  int bits, uint64_t n, float* acc, uint64_t bucket,
+                                  int add_into_acc, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    mqg::WorkerPtrs ptrs;
+    if (mqg_status st = check_workers(codes, scales, W, n == 0, &ptrs)) return st;
+    if (n == 0) return MQG_OK;
+    if (!acc) return fail(MQG_ERR_INVALID, "acc is null");
+    if (!aligned16(acc)) return fail(MQG_ERR_ALIGN, "acc not 16-byte aligned");
+    const cudaError_t err = mqg::launch_server(ptrs, W, bits, n, bucket, nullptr, 0.0f, acc,
+                                               add_into_acc ? 1 : 0,
+                                               static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_dequant_accumulate", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_apply(float* params, const float* acc, float lr, uint64_t n, void* cuda_stream)
+{
+    if (n == 0) return MQG_OK;
+    if (!params || !acc) return fail(MQG_ERR_INVALID, "params or acc is null");
+    if (!aligned16(params) || !aligned16(acc)) return fail(MQG_ERR_ALIGN, "params / acc not 16-byte aligned");
+    const cudaError_t err = mqg::launch_apply(params, acc, lr, n, static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_apply", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_server_step(const uint32_t* const* codes, const float* const* scales, int W, int bits,
+                           uint64_t n, uint64_t bucket, float* params, float lr, float* acc_out,
+                           void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    mqg::WorkerPtrs ptrs;
+    if (mqg_status st = check_workers(codes, scales, W, n == 0, &ptrs)) return st;
+    if (n == 0) return MQG_OK;
+    if (!params) return fail(MQG_ERR_INVALID, "params is null");
+    if (!aligned16(params)) return fail(MQG_ERR_ALIGN, "params not 16-byte aligned");
+    if (acc_out && !aligned16(acc_out)) return fail(MQG_ERR_ALIGN, "acc_out not 16-byte aligned");
+    const cudaError_t err = mqg::launch_server(ptrs, W, bits, n, bucket, params, lr, acc_out, 0,
+                                               static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_server_step", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg_off,
+                                 const uint64_t* code_off, int bits, uint64_t seed,
+                                 uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                                 uint32_t step, uint64_t elem_offset, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (nseg > 0) {
+        if (!grad || !codes || !scales) return fail(MQG_ERR_INVALID, "grad, codes or scales is null");
+        if (!aligned16(grad)) return fail(MQG_ERR_ALIGN, "grad not 16-byte aligned");
+        if (!aligned16(codes)) return fail(MQG_ERR_ALIGN, "codes not 16-byte aligned");
+        if (!aligned4(scales)) return fail(MQG_ERR_ALIGN, "scales not 4-byte aligned");
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            const cudaError_t err = mqg::launch_quantize_segments(grad, tab, bits, seed, codes,
+                                                                  scales + first, (int)dtype, worker,
+                                                                  step, elem_offset, stream);
+            if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments", err);
+            return MQG_OK;
+        });
+}
+
+mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* const* scales, int W,
+                                    int bits, int nseg, const uint64_t* seg_off,
+                                    const uint64_t* code_off, float* params, float lr,
+                                    float* acc_out, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    mqg::WorkerPtrs ptrs;
+    if (mqg_status st = check_workers(codes, scales, W, nseg <= 0, &ptrs)) return st;
+    if (nseg > 0) {
+        if (!params) return fail(MQG_ERR_INVALID, "params is null");
+        if (!aligned16(params)) return fail(MQG_ERR_ALIGN, "params not 16-byte aligned");
+        if (acc_out && !aligned16(acc_out)) return fail(MQG_ERR_ALIGN, "acc_out not 16-byte aligned");
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            const cudaError_t err = mqg::launch_server_segments(ptrs, W, bits, tab, first, params,
+                                                                lr, acc_out, stream);
+            if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
+            return MQG_OK;
+        });
+}
+
+}  // extern "C"

@@ -1,0 +1,353 @@
+// Device-side building blocks shared by the libmqgrad kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mqg {
+
+// One thread owns one "row": 32 consecutive elements.  For every bit width K a row packs
+// into exactly K 32-bit words, so all shifts are compile-time constants and no code
+// straddles a thread boundary.
+constexpr int kRowElems = 32;
+constexpr int kMaxTileRows = 256;                 // rows per CTA tile = threads per CTA
+constexpr int kMaxFusedBucket = kRowElems * kMaxTileRows;   // largest bucket of the one-pass kernel
+
+// Scales below this are flushed to zero (2^-96).
+__device__ __forceinline__ float flush_limit() { return __uint_as_float(0x0F800000u); }
+
+// ---------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  Counter (c0..c3), key (k0,k1) -> four words.
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&y)[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    y[0] = c0; y[1] = c1; y[2] = c2; y[3] = c3;
+}
+
+struct DrawKey {
+    uint32_t seed_lo, seed_hi, worker, step;
+};
+
+// The 16-bit draws of the 32 elements at flat positions g0 .. g0+31, g0 % 8 == 0:
+// four Philox blocks, block index g >> 3; element g takes half (g & 1) of word (g & 7) >> 1.
+// h[j] holds the two draws of elements 2j (low half) and 2j+1 (high half).
+__device__ __forceinline__ void draw_row_aligned(uint64_t g0, const DrawKey& key, uint32_t (&h)[16])
+{
+    const uint64_t blk0 = g0 >> 3;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        const uint64_t blk = blk0 + b;
+        uint32_t y[4];
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), key.worker, key.step,
+                      key.seed_lo, key.seed_hi, y);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) h[4 * b + k] = y[k];
+    }
+}
+
+// Same for any g0 (slow path: up to five blocks, run-time selection).
+static __device__ __noinline__ void draw_row_unaligned(uint64_t g0, const DrawKey& key, uint32_t (&h)[16])
+{
+    uint32_t y[20];
+    const uint64_t blk0 = g0 >> 3;
+    for (int b = 0; b < 5; ++b) {
+        const uint64_t blk = blk0 + b;
+        uint32_t t[4];
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), key.worker, key.step,
+                      key.seed_lo, key.seed_hi, t);
+        for (int k = 0; k < 4; ++k) y[4 * b + k] = t[k];
+    }
+    const unsigned shift = (unsigned)(g0 & 7u);       // first element's field in the 40-field run
+    for (int j = 0; j < 16; ++j) {
+        const unsigned f0 = shift + 2u * j, f1 = f0 + 1u;
+        const uint32_t lo = (y[f0 >> 1] >> (16u * (f0 & 1u))) & 0xFFFFu;
+        const uint32_t hi = (y[f1 >> 1] >> (16u * (f1 & 1u))) & 0xFFFFu;
+        h[j] = lo | (hi << 16);
+    }
+}
+
+// Per-bucket encode constants: t = fma(x, inv, half_l).  A flushed bucket uses (0, 0), which
+// sends every finite x to t = 0 and therefore to code 0.
+struct EncodeScale {
+    float inv, half_l;
+};
+
+template <int BITS>
+__device__ __forceinline__ EncodeScale encode_scale(float s)
+{
+    constexpr float Lf = (float)((1 << BITS) - 1);
+    EncodeScale e;
+    if (s == 0.0f) { e.inv = 0.0f; e.half_l = 0.0f; }
+    else { e.inv = __fdiv_rn(Lf, __fmul_rn(2.0f, s)); e.half_l = 0.5f * Lf; }
+    return e;
+}
+
+// Stochastic-rounding code of one element.  h16 is the element's 16-bit draw.
+template <int BITS>
+__device__ __forceinline__ uint32_t encode_one(float x, const EncodeScale& e, uint32_t h16)
+{
+    constexpr float Lf = (float)((1 << BITS) - 1);
+    float t = __fmaf_rn(x, e.inv, e.half_l);
+    t = fminf(fmaxf(t, 0.0f), Lf);
+    const float f = floorf(t);
+    const float r = __fsub_rn(t, f);
+    const float u = __fmul_rn(__fadd_rn((float)h16, 0.5f), 1.0f / 65536.0f);
+    return (uint32_t)(int)f + ((u < r) ? 1u : 0u);
+}
+
+// Pack the 32 codes of a row, code j at bits [j*BITS, j*BITS+BITS), into BITS words.
+template <int BITS>
+__device__ __forceinline__ void pack_row(const uint32_t (&q)[32], uint32_t (&w)[BITS])
+{
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) w[k] = 0u;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int o = j * BITS, wi = o >> 5, sh = o & 31;
+        w[wi] |= q[j] << sh;
+        if (sh + BITS > 32) w[wi + 1] |= q[j] >> (32 - sh);
+    }
+}
+
+// Code j of a row from its BITS words.
+template <int BITS>
+__device__ __forceinline__ uint32_t unpack_one(const uint32_t (&w)[BITS], int j)
+{
+    const int o = j * BITS, wi = o >> 5, sh = o & 31;
+    uint32_t v = w[wi] >> sh;
+    if (sh + BITS > 32) v |= w[wi + 1] << (32 - sh);
+    return v & ((1u << BITS) - 1u);
+}
+
+// Zero the bits of a row's words at and beyond `valid_bits` (ragged last row).
+template <int BITS>
+__device__ __forceinline__ void mask_row_words(uint32_t (&w)[BITS], int valid_bits)
+{
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) {
+        const int rem = valid_bits - 32 * k;
+        if (rem <= 0) w[k] = 0u;
+        else if (rem < 32) w[k] &= (1u << rem) - 1u;
+    }
+}
+
+// Store / load the BITS words of a row at word index `word0` (a multiple of BITS), using the
+// widest access the alignment of every row allows.  `nwords_limit` guards a ragged last row.
+template <int BITS>
+__device__ __forceinline__ void store_row_words(uint32_t* __restrict__ codes, uint64_t word0,
+                                                const uint32_t (&w)[BITS])
+{
+    if constexpr (BITS % 4 == 0) {
+        uint4* p = reinterpret_cast<uint4*>(codes + word0);
+#pragma unroll
+        for (int k = 0; k < BITS / 4; ++k) p[k] = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+    } else if constexpr (BITS % 2 == 0) {
+        uint2* p = reinterpret_cast<uint2*>(codes + word0);
+#pragma unroll
+        for (int k = 0; k < BITS / 2; ++k) p[k] = make_uint2(w[2 * k], w[2 * k + 1]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < BITS; ++k) codes[word0 + k] = w[k];
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void load_row_words(const uint32_t* __restrict__ codes, uint64_t word0,
+                                               uint32_t (&w)[BITS])
+{
+    if constexpr (BITS % 4 == 0) {
+        const uint4* p = reinterpret_cast<const uint4*>(codes + word0);
+#pragma unroll
+        for (int k = 0; k < BITS / 4; ++k) {
+            const uint4 v = __ldg(p + k);
+            w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
+        }
+    } else if constexpr (BITS % 2 == 0) {
+        const uint2* p = reinterpret_cast<const uint2*>(codes + word0);
+#pragma unroll
+        for (int k = 0; k < BITS / 2; ++k) {
+            const uint2 v = __ldg(p + k);
+            w[2 * k] = v.x; w[2 * k + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < BITS; ++k) w[k] = __ldg(codes + word0 + k);
+    }
+}
+
+// Shared-memory tile of rows x 32 floats with the 128-byte swizzle: the 16-byte chunk c of
+// row r lives at chunk position c ^ (r & 7), so that eight threads reading the same chunk
+// index of eight consecutive rows touch all 32 banks.
+__device__ __forceinline__ int swz(int row, int chunk) { return row * 8 + (chunk ^ (row & 7)); }
+
+__device__ __forceinline__ void read_row(const float4* tile, int row, float (&x)[32])
+{
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const float4 v = tile[swz(row, c)];
+        x[4 * c] = v.x; x[4 * c + 1] = v.y; x[4 * c + 2] = v.z; x[4 * c + 3] = v.w;
+    }
+}
+
+__device__ __forceinline__ void write_row(float4* tile, int row, const float (&x)[32])
+{
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        tile[swz(row, c)] = make_float4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
+}
+
+// Cooperative, coalesced copy of a tile of `rows` rows into / out of a swizzled tile.  `src`
+// points at the tile's first element and `valid` is the number of elements that exist from
+// there on (elements at or beyond it read as zero and are never written).  128-bit accesses
+// when the tile's first element is 16-byte aligned, 32-bit (16-bit for bf16) otherwise.
+template <int THREADS>
+__device__ __forceinline__ void load_tile_f32(float4* tile, const float* __restrict__ src,
+                                              uint64_t valid, int rows)
+{
+    if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+        const int chunks = rows * 8;
+        for (int idx = threadIdx.x; idx < chunks; idx += THREADS) {
+            const uint64_t e = 4ull * idx;
+            float4 v;
+            if (e + 4 <= valid) v = __ldcs(reinterpret_cast<const float4*>(src + e));
+            else {
+                v.x = (e + 0 < valid) ? src[e + 0] : 0.0f;
+                v.y = (e + 1 < valid) ? src[e + 1] : 0.0f;
+                v.z = (e + 2 < valid) ? src[e + 2] : 0.0f;
+                v.w = 0.0f;
+            }
+            tile[swz(idx >> 3, idx & 7)] = v;
+        }
+    } else {
+        float* tf = reinterpret_cast<float*>(tile);
+        const int elems = rows * 32;
+        for (int k = threadIdx.x; k < elems; k += THREADS) {
+            const float v = ((uint64_t)k < valid) ? __ldcs(src + k) : 0.0f;
+            tf[swz(k >> 5, (k >> 2) & 7) * 4 + (k & 3)] = v;
+        }
+    }
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+template <int THREADS>
+__device__ __forceinline__ void load_tile_bf16(float4* tile, const uint16_t* __restrict__ src,
+                                               uint64_t valid, int rows)
+{
+    if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+        const int groups = rows * 4;                    // 8 bf16 (16 bytes) per group
+        for (int idx = threadIdx.x; idx < groups; idx += THREADS) {
+            const uint64_t e = 8ull * idx;
+            uint32_t u[4];
+            if (e + 8 <= valid) {
+                const uint4 v = __ldcs(reinterpret_cast<const uint4*>(src + e));
+                u[0] = v.x; u[1] = v.y; u[2] = v.z; u[3] = v.w;
+            } else {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t lo = (e + 2 * k < valid) ? src[e + 2 * k] : 0u;
+                    const uint32_t hi = (e + 2 * k + 1 < valid) ? src[e + 2 * k + 1] : 0u;
+                    u[k] = lo | (hi << 16);
+                }
+            }
+            const int row = idx >> 2, c = (idx & 3) * 2;
+            tile[swz(row, c)] = make_float4(bf16_lo(u[0]), bf16_hi(u[0]), bf16_lo(u[1]), bf16_hi(u[1]));
+            tile[swz(row, c + 1)] = make_float4(bf16_lo(u[2]), bf16_hi(u[2]), bf16_lo(u[3]), bf16_hi(u[3]));
+        }
+    } else {
+        float* tf = reinterpret_cast<float*>(tile);
+        const int elems = rows * 32;
+        for (int k = threadIdx.x; k < elems; k += THREADS) {
+            const uint32_t b = ((uint64_t)k < valid) ? (uint32_t)src[k] : 0u;
+            tf[swz(k >> 5, (k >> 2) & 7) * 4 + (k & 3)] = bf16_lo(b);
+        }
+    }
+}
+
+template <int THREADS>
+__device__ __forceinline__ void store_tile_f32(const float4* tile, float* __restrict__ dst,
+                                               uint64_t valid, int rows)
+{
+    if ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        const int chunks = rows * 8;
+        for (int idx = threadIdx.x; idx < chunks; idx += THREADS) {
+            const uint64_t e = 4ull * idx;
+            if (e >= valid) continue;
+            const float4 v = tile[swz(idx >> 3, idx & 7)];
+            if (e + 4 <= valid) *reinterpret_cast<float4*>(dst + e) = v;
+            else {
+                dst[e] = v.x;
+                if (e + 1 < valid) dst[e + 1] = v.y;
+                if (e + 2 < valid) dst[e + 2] = v.z;
+            }
+        }
+    } else {
+        const float* tf = reinterpret_cast<const float*>(tile);
+        const int elems = rows * 32;
+        for (int k = threadIdx.x; k < elems; k += THREADS)
+            if ((uint64_t)k < valid) dst[k] = tf[swz(k >> 5, (k >> 2) & 7) * 4 + (k & 3)];
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// De-quantization.  Constants of one (worker, bucket): x^ = fma(q - (L-1)/2, 2h, -h) with
+// h = fl(s / L).  The product (q - (L-1)/2) * 2h and the subtraction of h are exact inside
+// the fma, so its single rounding is the rounding of (2q - L) * h.  A zero scale gives +0.
+// ---------------------------------------------------------------------------------
+struct DecodeScale {
+    float two_h, minus_h;
+};
+
+template <int BITS>
+__device__ __forceinline__ DecodeScale decode_scale(float s)
+{
+    constexpr float Lf = (float)((1 << BITS) - 1);
+    DecodeScale d;
+    if (s == 0.0f) { d.two_h = 0.0f; d.minus_h = 0.0f; }
+    else {
+        const float h = __fdiv_rn(s, Lf);
+        d.two_h = __fmul_rn(2.0f, h);
+        d.minus_h = -h;
+    }
+    return d;
+}
+
+template <int BITS>
+__device__ __forceinline__ float decode_one(uint32_t q, const DecodeScale& d)
+{
+    constexpr float kHalf = (float)(((1 << BITS) - 2) / 2);      // (L - 1) / 2, an integer
+    const float qi = __fsub_rn((float)q, kHalf);
+    return __fmaf_rn(qi, d.two_h, d.minus_h);
+}
+
+// v[] <- v[] + de-quantized row (or v[] <- de-quantized row when `first`).
+template <int BITS>
+__device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const DecodeScale& d,
+                                                bool first, float (&v)[32])
+{
+    if (first) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = decode_one<BITS>(unpack_one<BITS>(w, j), d);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            v[j] = __fadd_rn(v[j], decode_one<BITS>(unpack_one<BITS>(w, j), d));
+    }
+}
+
+}  // namespace mqg

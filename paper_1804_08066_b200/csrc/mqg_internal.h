@@ -1,0 +1,61 @@
+// Host-side launchers behind the C ABI (arguments already validated by mqg_api.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mqg {
+
+constexpr int kMaxWorkers = 32;
+constexpr int kMaxSegmentsPerLaunch = 64;
+
+struct WorkerPtrs {
+    const uint32_t* codes[kMaxWorkers];
+    const float* scales[kMaxWorkers];
+};
+
+// Segment table passed by value to the segment kernels (one chunk of <= kMaxSegmentsPerLaunch
+// segments per launch).  A tile is 256 rows of 32 elements inside one segment.
+// uniform_bucket != 0 selects the arithmetic layout instead of the table: segment j is
+// elements [j * uniform_bucket, min((j+1) * uniform_bucket, n_total)), its codes start at word
+// j * uniform_bucket * bits / 32, and it has tiles_per_bucket tiles.
+struct SegmentTable {
+    int nseg;
+    uint32_t tile_start[kMaxSegmentsPerLaunch + 1];   // prefix sum of tiles per segment
+    uint64_t seg_off[kMaxSegmentsPerLaunch + 1];      // element offsets
+    uint64_t code_off[kMaxSegmentsPerLaunch];         // word offsets
+    uint64_t uniform_bucket;
+    uint64_t n_total;
+    uint32_t tiles_per_bucket;
+};
+
+cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64_t bucket,
+                                  uint64_t seed, uint32_t* codes, float* scales, int dtype,
+                                  uint32_t worker, uint32_t step, uint64_t elem_offset,
+                                  cudaStream_t stream);
+
+// Two-pass quantize of segments.  scales_base points at the scale of the table's first segment.
+cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, int bits,
+                                     uint64_t seed, uint32_t* codes, float* scales_base, int dtype,
+                                     uint32_t worker, uint32_t step, uint64_t elem_offset,
+                                     cudaStream_t stream);
+
+// Two-pass quantize with uniform large buckets (bucket > kMaxFusedBucket, or a single bucket
+// whose length is not a multiple of 32).
+cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, uint64_t bucket,
+                                        uint64_t seed, uint32_t* codes, float* scales, int dtype,
+                                        uint32_t worker, uint32_t step, uint64_t elem_offset,
+                                        cudaStream_t stream);
+
+// Server pass over uniform buckets.  params == nullptr: only accumulate (acc required).
+// params != nullptr: update params (acc optional output).  add_into only without params.
+cudaError_t launch_server(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                          float* params, float lr, float* acc, int add_into, cudaStream_t stream);
+
+cudaError_t launch_server_segments(const WorkerPtrs& ptrs, int W, int bits, const SegmentTable& tab,
+                                   int scale_base, float* params, float lr, float* acc,
+                                   cudaStream_t stream);
+
+cudaError_t launch_apply(float* params, const float* acc, float lr, uint64_t n, cudaStream_t stream);
+
+}  // namespace mqg

@@ -38,7 +38,8 @@ def normal(n: int, sigma: float, config: int = 1, worker: int = 0) -> np.ndarray
 def laplace(n: int, scale: float, config: int = 2, worker: int = 0) -> np.ndarray:
     """iid Laplace(0, scale) as float32, by the inverse CDF of a uniform."""
     u = _rng(config, worker).random(n, dtype=np.float32) - np.float32(0.5)
-    mag = -np.log1p(-2.0 * np.abs(u).astype(np.float64)).astype(np.float32)
+    a = np.minimum(2.0 * np.abs(u).astype(np.float64), 1.0 - 2.0 ** -24)   # keep the log finite
+    mag = (-np.log1p(-a)).astype(np.float32)
     return (np.sign(u) * mag * np.float32(scale)).astype(np.float32)
 
 
