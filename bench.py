@@ -407,6 +407,56 @@ def run_ours(args):
     return 0
 
 
+def run_single_kernel(args):
+    """A few launches of one kernel on a small case (inputs still larger than L2), for profiler
+    captures and quick timing: python bench.py --kernel quantize|server --bits B [--n N]."""
+    import torch
+
+    import paper_1804_08066_b200 as mqg
+    from paper_1804_08066_b200 import workloads as wl
+
+    torch.cuda.set_device(0)
+    n, W, B, b = args.n, args.workers, args.bucket, args.bits
+    rot = 3                                    # rotate buffer sets so launches never re-read L2
+    stream = torch.cuda.current_stream()
+    if args.kernel == "quantize":
+        grads = [torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w)).cuda() for w in range(rot)]
+        codes = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
+        scales = [torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize(grads[i % rot], n, b, B, PHILOX_SEED, codes[i % rot],
+                                            scales[i % rot], worker=i % rot, step=i)
+        nbytes = quantize_bytes(n, b, B)
+    else:
+        g = torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=0)).cuda()
+        codes = [[torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(W)]
+                 for _ in range(rot)]
+        scales = [[torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(W)]
+                  for _ in range(rot)]
+        for r in range(rot):
+            for w in range(W):
+                mqg.mqg_quantize(g, n, b, B, PHILOX_SEED, codes[r][w], scales[r][w], worker=w, step=r)
+        params = [torch.from_numpy(wl.params(n, 0.05, config=2)).cuda() for _ in range(rot)]
+        launch = lambda i: mqg.mqg_server_step(codes[i % rot], scales[i % rot], W, b, n, B,
+                                               params[i % rot], LR)
+        nbytes = server_bytes(n, b, B, W)
+    torch.cuda.synchronize()
+    times = []
+    for i in range(args.launches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        launch(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e-3)
+    peak, kind = measured_hbm_peak()
+    best, med = min(times), float(np.median(times))
+    print(json.dumps({"kernel": args.kernel, "bits": b, "n": n, "workers": W, "bucket": B,
+                      "launches": args.launches, "median_us": med * 1e6, "best_us": best * 1e6,
+                      "algorithmic_bytes": nbytes, "median_gbs": nbytes / med / 1e9,
+                      "frac_of_%s_peak" % kind: nbytes / med / 1e9 / peak}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -414,7 +464,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", choices=["quantize", "server"], default=None,
+                    help="run a few launches of one kernel on a small case instead of the benchmark")
+    ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--n", type=int, default=1 << 25)
+    ap.add_argument("--workers", type=int, default=N_WORKERS)
+    ap.add_argument("--bucket", type=int, default=BUCKET)
+    ap.add_argument("--launches", type=int, default=6)
     args = ap.parse_args()
+    if args.kernel is not None:
+        return run_single_kernel(args)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

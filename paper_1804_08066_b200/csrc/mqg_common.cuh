@@ -80,10 +80,11 @@ static __device__ __noinline__ void draw_row_unaligned(uint64_t g0, const DrawKe
     }
 }
 
-// Per-bucket encode constants: t = fma(x, inv, half_l).  A flushed bucket uses (0, 0), which
-// sends every finite x to t = 0 and therefore to code 0.
+// Per-bucket encode constants, pre-scaled by 2^16: T = fma(x, inv16, half_l16) = 2^16 * t with
+// t = fl(x * fl(L / 2s) + L/2) -- scaling both constants by a power of two leaves the single
+// rounding of the fma unchanged.  A flushed bucket uses (0, 0): every x gives T = 0, code 0.
 struct EncodeScale {
-    float inv, half_l;
+    float inv16, half_l16;
 };
 
 template <int BITS>
@@ -91,36 +92,60 @@ __device__ __forceinline__ EncodeScale encode_scale(float s)
 {
     constexpr float Lf = (float)((1 << BITS) - 1);
     EncodeScale e;
-    if (s == 0.0f) { e.inv = 0.0f; e.half_l = 0.0f; }
-    else { e.inv = __fdiv_rn(Lf, __fmul_rn(2.0f, s)); e.half_l = 0.5f * Lf; }
+    if (s == 0.0f) { e.inv16 = 0.0f; e.half_l16 = 0.0f; }
+    else {
+        e.inv16 = __fmul_rn(__fdiv_rn(Lf, __fmul_rn(2.0f, s)), 65536.0f);
+        e.half_l16 = 32768.0f * Lf;
+    }
     return e;
 }
 
-// Stochastic-rounding code of one element.  h16 is the element's 16-bit draw.
-template <int BITS>
-__device__ __forceinline__ uint32_t encode_one(float x, const EncodeScale& e, uint32_t h16)
+// Stochastic-rounding code of one element, as the bit pattern of the float 1.5 * 2^23 + q.
+// `hf` is the float 2^23 + h (h = the element's 16-bit draw, merged into the mantissa).
+//   code = floor(t) + [u < t - floor(t)],  u = (h + 1/2) / 2^16
+//        = ceil(t - u) = ceil((T - (h + 1/2)) / 2^16).
+// |T| stands for the clamp to [0, L]: t <= L always holds for |x| <= s, and a t rounded
+// slightly below zero has |t| < 2^-17 <= u, which gives code 0 like the clamp.
+// Rounding the difference up cannot cross a multiple of 2^16 (those are floats), and adding
+// 1.5 * 2^23 with rounding up leaves the ceiling in the low mantissa bits.
+__device__ __forceinline__ uint32_t encode_bits(float x, const EncodeScale& e, float hf)
 {
-    constexpr float Lf = (float)((1 << BITS) - 1);
-    float t = __fmaf_rn(x, e.inv, e.half_l);
-    t = fminf(fmaxf(t, 0.0f), Lf);
-    const float f = floorf(t);
-    const float r = __fsub_rn(t, f);
-    const float u = __fmul_rn(__fadd_rn((float)h16, 0.5f), 1.0f / 65536.0f);
-    return (uint32_t)(int)f + ((u < r) ? 1u : 0u);
+    const float T = __fmaf_rn(x, e.inv16, e.half_l16);
+    const float hh = __fsub_rn(hf, 8388607.5f);                 // h + 1/2, exact
+    const float d = __fadd_ru(fabsf(T), -hh);
+    const float w = __fmaf_ru(d, 1.0f / 65536.0f, 12582912.0f);
+    return __float_as_uint(w);
 }
+constexpr uint32_t kCodeBias = 0x4B400000u;      // bit pattern of 1.5 * 2^23
 
-// Pack the 32 codes of a row, code j at bits [j*BITS, j*BITS+BITS), into BITS words.
+// 2^23 + h for the low / high 16-bit half of a Philox word.
+__device__ __forceinline__ float draw_lo(uint32_t y) { return __uint_as_float(__byte_perm(y, 0x4B000000u, 0x7610)); }
+__device__ __forceinline__ float draw_hi(uint32_t y) { return __uint_as_float(__byte_perm(y, 0x4B000000u, 0x7632)); }
+
+// Encode the 32 values of a row and pack them, code j at bits [j*BITS, j*BITS+BITS), into BITS
+// words.  The biased patterns kCodeBias + q are accumulated with multiply-adds; the bias
+// contributions are compile-time constants removed at the end.
 template <int BITS>
-__device__ __forceinline__ void pack_row(const uint32_t (&q)[32], uint32_t (&w)[BITS])
+__device__ __forceinline__ void encode_pack_row(const float (&x)[32], const EncodeScale& e,
+                                                const uint32_t (&h)[16], uint32_t (&w)[BITS])
 {
+    uint32_t bias[BITS];
 #pragma unroll
-    for (int k = 0; k < BITS; ++k) w[k] = 0u;
+    for (int k = 0; k < BITS; ++k) { w[k] = 0u; bias[k] = 0u; }
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
+        const float hf = (j & 1) ? draw_hi(h[j >> 1]) : draw_lo(h[j >> 1]);
+        const uint32_t c = encode_bits(x[j], e, hf);
         const int o = j * BITS, wi = o >> 5, sh = o & 31;
-        w[wi] |= q[j] << sh;
-        if (sh + BITS > 32) w[wi + 1] |= q[j] >> (32 - sh);
+        w[wi] += c << sh;
+        bias[wi] += kCodeBias << sh;
+        if (sh + BITS > 32) {
+            w[wi + 1] += c >> (32 - sh);          // the bias has 22 zero low bits: no carry mixes in
+            bias[wi + 1] += kCodeBias >> (32 - sh);
+        }
     }
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) w[k] -= bias[k];
 }
 
 // Code j of a row from its BITS words.
@@ -327,26 +352,65 @@ __device__ __forceinline__ DecodeScale decode_scale(float s)
     return d;
 }
 
+// m = the float 2^23 + q (code merged into the mantissa of 2^23).
 template <int BITS>
-__device__ __forceinline__ float decode_one(uint32_t q, const DecodeScale& d)
+__device__ __forceinline__ float decode_biased(float m, const DecodeScale& d)
 {
-    constexpr float kHalf = (float)(((1 << BITS) - 2) / 2);      // (L - 1) / 2, an integer
-    const float qi = __fsub_rn((float)q, kHalf);
-    return __fmaf_rn(qi, d.two_h, d.minus_h);
+    constexpr float kOff = 8388608.0f + (float)(((1 << BITS) - 2) / 2);   // 2^23 + (L - 1) / 2
+    return __fmaf_rn(__fsub_rn(m, kOff), d.two_h, d.minus_h);
 }
 
-// v[] <- v[] + de-quantized row (or v[] <- de-quantized row when `first`).
+__device__ __forceinline__ float byte_to_biased(uint32_t v, int byte)
+{
+    return __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7650 + byte));
+}
+
+// v[] <- v[] + de-quantized row, v must hold the running sum (+0 before the first worker:
+// 0 + x^ is exact, and turns the -0 of a zero-scale bucket into +0).
 template <int BITS>
 __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const DecodeScale& d,
-                                                bool first, float (&v)[32])
+                                                float (&v)[32])
 {
-    if (first) {
+    if constexpr (BITS == 1) {
+        // x^ = +-s: flip the sign of s (= 2h - h... h itself) where the code bit is 0
+        const uint32_t sbits = __float_as_uint(-d.minus_h);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = decode_one<BITS>(unpack_one<BITS>(w, j), d);
-    } else {
+        for (int j = 0; j < 32; ++j) {
+            const uint32_t sign = (~(w[0] << (31 - j))) & 0x80000000u;
+            v[j] = __fadd_rn(v[j], __uint_as_float(sbits | sign));
+        }
+    } else if constexpr (BITS == 8) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)
-            v[j] = __fadd_rn(v[j], decode_one<BITS>(unpack_one<BITS>(w, j), d));
+            v[j] = __fadd_rn(v[j], decode_biased<8>(byte_to_biased(w[j >> 2], j & 3), d));
+    } else if constexpr (BITS == 4) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                v[8 * k + 2 * b] = __fadd_rn(v[8 * k + 2 * b], decode_biased<4>(byte_to_biased(lo, b), d));
+                v[8 * k + 2 * b + 1] = __fadd_rn(v[8 * k + 2 * b + 1], decode_biased<4>(byte_to_biased(hi, b), d));
+            }
+        }
+    } else if constexpr (BITS == 2) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const uint32_t t = (w[k] >> (2 * r)) & 0x03030303u;
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    v[16 * k + 4 * b + r] = __fadd_rn(v[16 * k + 4 * b + r],
+                                                      decode_biased<2>(byte_to_biased(t, b), d));
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const uint32_t q = unpack_one<BITS>(w, j);
+            v[j] = __fadd_rn(v[j], decode_biased<BITS>(__uint_as_float(q | 0x4B000000u), d));
+        }
     }
 }
 

@@ -98,14 +98,8 @@ quantize_pack_kernel(const QuantizeArgs a)
     if constexpr (ALIGNED_DRAWS) draw_row_aligned(a.elem_offset + row * 32, a.key, h);
     else draw_row_unaligned(a.elem_offset + row * 32, a.key, h);
 
-    uint32_t q[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const uint32_t h16 = (j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu);
-        q[j] = encode_one<BITS>(x[j], es, h16);
-    }
     uint32_t w[BITS];
-    pack_row<BITS>(q, w);
+    encode_pack_row<BITS>(x, es, h, w);
 
     const uint64_t word0 = row * BITS;
     const uint64_t e0 = row * 32;

@@ -96,14 +96,8 @@ encode_segments_kernel(const SegQuantArgs a, const SegmentTable tab)
     if ((g0 & 7u) == 0) draw_row_aligned(g0, a.key, h);
     else draw_row_unaligned(g0, a.key, h);
 
-    uint32_t q[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const uint32_t h16 = (j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu);
-        q[j] = encode_one<BITS>(x[j], es, h16);
-    }
     uint32_t w[BITS];
-    pack_row<BITS>(q, w);
+    encode_pack_row<BITS>(x, es, h, w);
 
     const uint64_t word0 = g.word0 + (uint64_t)t * BITS;
     const uint64_t left = g.valid - 32ull * t;          // elements of the segment from this row on

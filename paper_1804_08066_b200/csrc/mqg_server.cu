@@ -29,6 +29,10 @@ __device__ __forceinline__ void accumulate_row(const ServerArgs& a, uint64_t sca
                                                uint64_t word0, uint64_t words_end, bool full_row,
                                                float (&v)[32], bool have_init)
 {
+    if (!have_init) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+    }
     for (int wk = 0; wk < a.W; ++wk) {
         uint32_t w[BITS];
         if (VEC && full_row) load_row_words<BITS>(a.ptrs.codes[wk], word0, w);
@@ -38,7 +42,7 @@ __device__ __forceinline__ void accumulate_row(const ServerArgs& a, uint64_t sca
                 w[k] = (word0 + k < words_end) ? __ldg(a.ptrs.codes[wk] + word0 + k) : 0u;
         }
         const DecodeScale d = decode_scale<BITS>(__ldg(a.ptrs.scales[wk] + scale_idx));
-        add_decoded_row<BITS>(w, d, wk == 0 && !have_init, v);
+        add_decoded_row<BITS>(w, d, v);
     }
 }
 
