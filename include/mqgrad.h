@@ -134,6 +134,15 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
                                     const uint64_t* code_off, float* params, float lr,
                                     float* acc_out, void* cuda_stream);
 
+/*
+ * Kernels stage data through shared memory with asynchronous bulk copies and wait for them on
+ * barriers with a bounded number of polls; a wait that runs out makes the kernel record it in a
+ * per-device counter, abandon its work and return (its outputs are then incomplete) instead of
+ * hanging.  This call synchronises with the current device and stores the number of such events
+ * since the library was loaded in *count (0 in a healthy run).  Returns MQG_OK or MQG_ERR_CUDA.
+ */
+mqg_status mqg_device_timeouts(unsigned int* count);
+
 /* Message of the last error returned to the calling thread ("" if none).  Never NULL. */
 const char* mqg_last_error(void);
 

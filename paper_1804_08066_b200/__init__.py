@@ -8,7 +8,7 @@ raises.
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_quantize_segments, mqg_server_step_segments, mqg_code_words, mqg_num_buckets,
-  mqg_wire_bytes, mqg_last_error, mqg_version.
+  mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
 from __future__ import annotations
 
@@ -37,7 +37,7 @@ class MqgError(RuntimeError):
 def _load() -> C.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            "libmqgrad.so is not built (%s); run `python -m paper_1804_08066_b200.build`. "
+            "libmqgrad.so is not built (%s); run `python paper_1804_08066_b200/build.py`. "
             "There is no fallback path." % LIB_PATH)
     lib = C.CDLL(LIB_PATH)
     u64, u32, i32, vp, f32 = C.c_uint64, C.c_uint32, C.c_int, C.c_void_p, C.c_float
@@ -47,6 +47,7 @@ def _load() -> C.CDLL:
         "mqg_wire_bytes": (C.c_size_t, [u64, i32, u64]),
         "mqg_last_error": (C.c_char_p, []),
         "mqg_version": (i32, []),
+        "mqg_device_timeouts": (i32, [C.POINTER(C.c_uint)]),
         "mqg_quantize": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
         "mqg_apply": (i32, [vp, vp, f32, u64, vp]),
@@ -110,6 +111,13 @@ def mqg_last_error() -> str:
 
 def mqg_version() -> int:
     return int(_lib.mqg_version())
+
+
+def mqg_device_timeouts() -> int:
+    """Number of kernel waits that gave up on the current device (synchronises); 0 when healthy."""
+    c = C.c_uint(0)
+    _check(_lib.mqg_device_timeouts(C.byref(c)))
+    return int(c.value)
 
 
 def _grad_dtype(grad) -> int:

@@ -1,6 +1,6 @@
 """Build libmqgrad.so (sm_100a) in-tree with nvcc.
 
-Usage: python -m paper_1804_08066_b200.build [--force] [--verbose]
+Usage: python paper_1804_08066_b200/build.py [--force] [--verbose]
 The shared object lands next to this file; nvcc cross-compiles without a GPU.
 """
 import glob
@@ -15,7 +15,7 @@ LIB = os.path.join(HERE, "libmqgrad.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE,
+    "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "--threads", "4",
 ]
 
 

@@ -6,6 +6,7 @@
 #include "../../include/mqgrad.h"
 #include "mqg_common.cuh"
 #include "mqg_internal.h"
+#include "mqg_tma.cuh"
 
 namespace {
 
@@ -127,6 +128,14 @@ size_t mqg_wire_bytes(uint64_t n, int bits, uint64_t bucket)
 const char* mqg_last_error(void) { return g_err; }
 
 int mqg_version(void) { return 100; }
+
+mqg_status mqg_device_timeouts(unsigned int* count)
+{
+    if (!count) return fail(MQG_ERR_INVALID, "count is null");
+    const cudaError_t err = mqg::read_wait_timeouts(count);
+    if (err != cudaSuccess) return cuda_fail("mqg_device_timeouts", err);
+    return MQG_OK;
+}
 
 mqg_status mqg_quantize(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
                         uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,

@@ -9,6 +9,7 @@
 // from HBM exactly once.
 #include "mqg_common.cuh"
 #include "mqg_internal.h"
+#include "mqg_tma.cuh"
 
 namespace mqg {
 
@@ -24,6 +25,8 @@ struct QuantizeArgs {
     uint32_t rows_per_bucket;   // bucket / 32 (a single ragged bucket counts as "all rows")
     uint32_t tile_rows;         // rows per tile: a multiple of rows_per_bucket, <= 256
     uint32_t buckets_per_tile;
+    uint64_t nrows_full;    // floor(n / 32): rows the tensor map covers
+    uint32_t ntiles;
     DrawKey key;
 };
 
@@ -114,6 +117,169 @@ quantize_pack_kernel(const QuantizeArgs a)
     }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// The same computation fed by TMA: a persistent CTA walks tiles blockIdx.x, +gridDim.x, ...;
+// one elected thread keeps STAGES tiled bulk copies (cp.async.bulk.tensor, 128- or 64-byte
+// swizzle) in flight into a shared-memory ring, each completing on its own mbarrier, so the
+// compute warps never issue a global load and never wait for DRAM latency in steady state.
+// One __syncthreads per tile publishes the bucket maxima and releases the stage for refill.
+// ---------------------------------------------------------------------------------------
+template <int DTYPE>
+__device__ __forceinline__ void read_row_swizzled(const uint8_t* stage, int row, float (&x)[32])
+{
+    if constexpr (DTYPE == 0) {
+        read_row(reinterpret_cast<const float4*>(stage), row, x);
+    } else {
+        const uint4* t = reinterpret_cast<const uint4*>(stage);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint4 v = t[row * 4 + (c ^ ((row >> 1) & 3))];
+            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                x[8 * c + 2 * k] = bf16_lo(u[k]);
+                x[8 * c + 2 * k + 1] = bf16_hi(u[k]);
+            }
+        }
+    }
+}
+
+// The one row of the gradient that is shorter than 32 elements is not covered by the tensor
+// map: its owner copies it (zero-padded) into its own row of the stage with plain loads and
+// then reads it back like any other row.
+template <int DTYPE>
+__device__ __noinline__ void stage_ragged_row(uint8_t* stage, int row, const void* grad, uint64_t e0,
+                                              uint64_t n)
+{
+    for (int j = 0; j < 32; ++j) {
+        const bool in = e0 + j < n;
+        if constexpr (DTYPE == 0) {
+            float* tf = reinterpret_cast<float*>(stage);
+            tf[swz(row, j >> 2) * 4 + (j & 3)] = in ? static_cast<const float*>(grad)[e0 + j] : 0.0f;
+        } else {
+            uint16_t* th = reinterpret_cast<uint16_t*>(stage);
+            const int chunk = (j >> 3) ^ ((row >> 1) & 3);
+            th[(row * 4 + chunk) * 8 + (j & 7)] = in ? static_cast<const uint16_t*>(grad)[e0 + j] : (uint16_t)0;
+        }
+    }
+}
+
+template <int BITS, int DTYPE, int THREADS, int STAGES>
+__global__ void __launch_bounds__(THREADS)
+quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const QuantizeArgs a,
+                    unsigned int* __restrict__ timeouts)
+{
+    constexpr int ROW_BYTES = DTYPE == 0 ? 128 : 64;
+    constexpr int STAGE_BYTES = THREADS * ROW_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint32_t* slots = reinterpret_cast<uint32_t*>(base + STAGES * STAGE_BYTES);      // [3][THREADS]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(slots + 3 * THREADS);               // [STAGES]
+
+    const uint32_t t = threadIdx.x;
+    const uint32_t my_count = a.ntiles > blockIdx.x ? (a.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t box_bytes = a.tile_rows * ROW_BYTES;
+    const uint32_t rpb = a.rows_per_bucket;
+    const bool shuffle_only = (rpb & (rpb - 1)) == 0 && rpb <= 32;
+
+    if (t == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        fence_barrier_init();
+    }
+    for (int i = t; i < 3 * THREADS; i += THREADS) slots[i] = 0u;
+    __syncthreads();
+
+    auto issue = [&](uint32_t k) {
+        const int s = k % STAGES;
+        const uint32_t tile = blockIdx.x + k * gridDim.x;
+        const uint32_t bar = smem_u32(&bars[s]);
+        mbar_expect_tx(bar, box_bytes);
+        tma_load_2d(smem_u32(base + s * STAGE_BYTES), &tmap, 0, (int)(tile * a.tile_rows), bar);
+    };
+    if (t == 0) {
+        prefetch_tensormap(&tmap);
+        for (uint32_t k = 0; k < (uint32_t)STAGES && k < my_count; ++k) issue(k);
+    }
+
+    const uint32_t local_bucket = t / rpb;
+    const bool scale_writer = (t % rpb) == 0;
+    uint32_t k = 0;
+    bool failed = false;
+    for (; k < my_count; ++k) {
+        const int s = k % STAGES;
+        const uint32_t tile = blockIdx.x + k * gridDim.x;
+        const uint64_t row0 = (uint64_t)tile * a.tile_rows;
+        const uint64_t rows_left = a.nrows - row0;
+        const uint32_t rows = rows_left < a.tile_rows ? (uint32_t)rows_left : a.tile_rows;
+        const bool active = t < rows;
+        const uint64_t row = row0 + t;
+
+        const bool ok = mbar_wait(smem_u32(&bars[s]), (k / STAGES) & 1);
+
+        float x[32];
+        if (active) {
+            if (row >= a.nrows_full)
+                stage_ragged_row<DTYPE>(base + s * STAGE_BYTES, (int)t, a.grad, row * 32, a.n);
+            read_row_swizzled<DTYPE>(base + s * STAGE_BYTES, (int)t, x);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) x[j] = 0.0f;
+        }
+        float mx = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(x[j]));
+        uint32_t m = __float_as_uint(mx);
+
+        uint32_t* slot = slots + (k % 3) * THREADS;
+        if (shuffle_only) {
+            for (uint32_t d = rpb >> 1; d > 0; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+        } else {
+            m = __reduce_max_sync(0xFFFFFFFFu, m);        // rpb % 32 == 0: a warp is inside one bucket
+            if ((t & 31) == 0 && active) atomicMax(&slot[local_bucket], m);
+        }
+        failed = __syncthreads_or(!ok) != 0;
+        if (failed) break;
+        if (t == 0 && k + STAGES < my_count) issue(k + STAGES);      // every thread has read stage s
+        if (!shuffle_only) {
+            m = slot[local_bucket];
+            if (t < a.buckets_per_tile) slots[((k + 2) % 3) * THREADS + t] = 0u;   // next use: tile k + 2
+        }
+        if (!active) continue;
+
+        float sc = __uint_as_float(m);
+        if (sc < flush_limit()) sc = 0.0f;
+        const uint64_t bucket = (uint64_t)tile * a.buckets_per_tile + local_bucket;
+        if (scale_writer && bucket < a.nbuckets) a.scales[bucket] = sc;
+
+        const EncodeScale es = encode_scale<BITS>(sc);
+        uint32_t h[16];
+        draw_row_aligned(a.elem_offset + row * 32, a.key, h);
+        uint32_t w[BITS];
+        encode_pack_row<BITS>(x, es, h, w);
+
+        const uint64_t word0 = row * BITS;
+        if (row * 32 + 32 <= a.n) {
+            store_row_words<BITS>(a.codes, word0, w);
+        } else {
+            mask_row_words<BITS>(w, (int)(a.n - row * 32) * BITS);
+#pragma unroll
+            for (int j = 0; j < BITS; ++j)
+                if (word0 + j < a.ncode_words) a.codes[word0 + j] = w[j];
+        }
+    }
+    if (failed) {
+        // a copy never landed: record it, wait (bounded) for the copies still in flight so that
+        // none can write into shared memory after this CTA has gone, and leave
+        if (t == 0) {
+            atomicAdd(timeouts, 1u);
+            for (uint32_t j = k; j < my_count && j < k + STAGES; ++j)
+                mbar_wait(smem_u32(&bars[j % STAGES]), (j / STAGES) & 1);
+        }
+        __syncthreads();
+    }
+}
+
 template <int BITS>
 static cudaError_t launch_bits(const QuantizeArgs& a, int dtype, bool aligned, unsigned grid,
                                cudaStream_t stream)
@@ -127,6 +293,59 @@ static cudaError_t launch_bits(const QuantizeArgs& a, int dtype, bool aligned, u
         else quantize_pack_kernel<BITS, 1, false><<<g, b, 0, stream>>>(a);
     }
     return cudaGetLastError();
+}
+
+template <int BITS, int DTYPE, int THREADS>
+static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a, unsigned int* timeouts,
+                                   cudaStream_t stream)
+{
+    constexpr int STAGES = 3;
+    constexpr int ROW_BYTES = DTYPE == 0 ? 128 : 64;
+    constexpr size_t smem = 1024 + (size_t)STAGES * THREADS * ROW_BYTES + 3 * THREADS * 4 + STAGES * 8;
+    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, STAGES>;
+    static int ctas_per_sm[64] = {};               // per device; 0 = not yet configured
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    static int sm_count[64] = {};
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (ctas_per_sm[dev] == 0) {
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        int occ = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, THREADS, smem);
+        if (err != cudaSuccess) return err;
+        int sms = 0;
+        err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (err != cudaSuccess) return err;
+        sm_count[dev] = sms;
+        ctas_per_sm[dev] = occ > 0 ? occ : 1;
+    }
+    unsigned grid = (unsigned)sm_count[dev] * (unsigned)ctas_per_sm[dev];
+    if (grid > a.ntiles) grid = a.ntiles;
+    kernel<<<grid, THREADS, smem, stream>>>(map, a, timeouts);
+    return cudaGetLastError();
+}
+
+template <int BITS>
+static cudaError_t launch_tma_bits(const CUtensorMap& map, const QuantizeArgs& a, int dtype, int threads,
+                                   unsigned int* timeouts, cudaStream_t stream)
+{
+    if (dtype == 0) {
+        if (threads == 128) return launch_tma_inst<BITS, 0, 128>(map, a, timeouts, stream);
+        return launch_tma_inst<BITS, 0, 256>(map, a, timeouts, stream);
+    }
+    if (threads == 128) return launch_tma_inst<BITS, 1, 128>(map, a, timeouts, stream);
+    return launch_tma_inst<BITS, 1, 256>(map, a, timeouts, stream);
+}
+
+// TMA path: whole rows exist, draws are block-aligned, and a bucket is either an aligned
+// power-of-two group of at most 32 rows or a whole number of warps.
+static bool tma_path_applies(uint64_t n, uint64_t rpb, uint64_t elem_offset)
+{
+    if (n < 32 * 64 || (elem_offset & 7u) != 0 || rpb == 0 || rpb > (uint64_t)kMaxTileRows) return false;
+    if (n / 32 > 0x7FFFFFFFull) return false;
+    return ((rpb & (rpb - 1)) == 0 && rpb <= 32) || rpb % 32 == 0;
 }
 
 cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64_t bucket,
@@ -148,8 +367,38 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
     a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
     a.key.seed_lo = (uint32_t)seed; a.key.seed_hi = (uint32_t)(seed >> 32);
     a.key.worker = worker; a.key.step = step;
+    a.nrows_full = n / 32;
+    if (tma_path_applies(n, rpb, elem_offset)) {
+        const int threads = rpb <= 128 ? 128 : 256;
+        a.buckets_per_tile = (uint32_t)(threads / rpb);
+        a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
+        const uint64_t nt = (a.nrows + a.tile_rows - 1) / a.tile_rows;
+        if (nt > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+        a.ntiles = (uint32_t)nt;
+        CUtensorMap map;
+        const char* why = nullptr;
+        unsigned int* timeouts = wait_timeout_counter();
+        if (timeouts != nullptr &&
+            encode_rows_map(&map, grad, a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why)) {
+            switch (bits) {
+                case 1: return launch_tma_bits<1>(map, a, dtype, threads, timeouts, stream);
+                case 2: return launch_tma_bits<2>(map, a, dtype, threads, timeouts, stream);
+                case 3: return launch_tma_bits<3>(map, a, dtype, threads, timeouts, stream);
+                case 4: return launch_tma_bits<4>(map, a, dtype, threads, timeouts, stream);
+                case 5: return launch_tma_bits<5>(map, a, dtype, threads, timeouts, stream);
+                case 6: return launch_tma_bits<6>(map, a, dtype, threads, timeouts, stream);
+                case 7: return launch_tma_bits<7>(map, a, dtype, threads, timeouts, stream);
+                case 8: return launch_tma_bits<8>(map, a, dtype, threads, timeouts, stream);
+            }
+            return cudaErrorInvalidValue;
+        }
+        return cudaErrorNotSupported;        // the driver cannot encode a tensor map: no silent detour
+    }
+    a.buckets_per_tile = (uint32_t)(kMaxTileRows / rpb);
+    a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
     const uint64_t ntiles = (a.nrows + a.tile_rows - 1) / a.tile_rows;
     if (ntiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    a.ntiles = (uint32_t)ntiles;
     const bool aligned = (elem_offset & 7u) == 0;
     switch (bits) {
         case 1: return launch_bits<1>(a, dtype, aligned, (unsigned)ntiles, stream);

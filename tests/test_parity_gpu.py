@@ -19,6 +19,12 @@ pytestmark = pytest.mark.gpu
 ALL_BITS = list(range(1, 9))
 
 
+@pytest.fixture(autouse=True)
+def no_kernel_wait_gave_up():
+    yield
+    assert mqg.mqg_device_timeouts() == 0, "a kernel's bounded wait ran out"
+
+
 def gpu_quantize(x, bits, bucket, seed, worker=0, step=0, elem_offset=0, bf16=False):
     n = x.size
     if bf16:
