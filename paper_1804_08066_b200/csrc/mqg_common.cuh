@@ -18,57 +18,81 @@ __device__ __forceinline__ float flush_limit() { return __uint_as_float(0x0F8000
 
 // ---------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11).  Counter (c0..c3), key (k0,k1) -> four words.
+// The ten round keys depend only on the seed, so they are computed once per thread
+// (RoundKeys) and stay in registers across all blocks.
 // ---------------------------------------------------------------------------------
+struct DrawKey {
+    uint32_t seed_lo, seed_hi, worker, step;
+};
+
+struct RoundKeys {
+    uint32_t k0[10], k1[10];
+    uint32_t worker, step;
+};
+
+__device__ __forceinline__ RoundKeys make_round_keys(const DrawKey& key)
+{
+    RoundKeys rk;
+    uint32_t a = key.seed_lo, b = key.seed_hi;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        rk.k0[r] = a; rk.k1[r] = b;
+        a += 0x9E3779B9u; b += 0xBB67AE85u;
+    }
+    rk.worker = key.worker; rk.step = key.step;
+    return rk;
+}
+
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t (&y)[4])
+                                              const RoundKeys& rk, uint32_t (&y)[4])
 {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
         const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
-        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k1[r];
         c1 = (uint32_t)p1;
         c3 = (uint32_t)p0;
         c0 = n0;
         c2 = n2;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     y[0] = c0; y[1] = c1; y[2] = c2; y[3] = c3;
 }
 
-struct DrawKey {
-    uint32_t seed_lo, seed_hi, worker, step;
-};
-
 // The 16-bit draws of the 32 elements at flat positions g0 .. g0+31, g0 % 8 == 0:
 // four Philox blocks, block index g >> 3; element g takes half (g & 1) of word (g & 7) >> 1.
 // h[j] holds the two draws of elements 2j (low half) and 2j+1 (high half).
-__device__ __forceinline__ void draw_row_aligned(uint64_t g0, const DrawKey& key, uint32_t (&h)[16])
+// (blk_lo, blk_hi) = 64-bit block index of the row's first element.
+__device__ __forceinline__ void draw_row_blocks(uint32_t blk_lo, uint32_t blk_hi, const RoundKeys& rk,
+                                                uint32_t (&h)[16])
 {
-    const uint64_t blk0 = g0 >> 3;
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
-        const uint64_t blk = blk0 + b;
         uint32_t y[4];
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), key.worker, key.step,
-                      key.seed_lo, key.seed_hi, y);
+        const uint32_t lo = blk_lo + b;
+        philox4x32_10(lo, blk_hi + (lo < blk_lo ? 1u : 0u), rk.worker, rk.step, rk, y);
 #pragma unroll
         for (int k = 0; k < 4; ++k) h[4 * b + k] = y[k];
     }
 }
 
+__device__ __forceinline__ void draw_row_aligned(uint64_t g0, const RoundKeys& rk, uint32_t (&h)[16])
+{
+    const uint64_t blk0 = g0 >> 3;
+    draw_row_blocks((uint32_t)blk0, (uint32_t)(blk0 >> 32), rk, h);
+}
+
 // Same for any g0 (slow path: up to five blocks, run-time selection).
 static __device__ __noinline__ void draw_row_unaligned(uint64_t g0, const DrawKey& key, uint32_t (&h)[16])
 {
+    const RoundKeys rk = make_round_keys(key);
     uint32_t y[20];
     const uint64_t blk0 = g0 >> 3;
     for (int b = 0; b < 5; ++b) {
         const uint64_t blk = blk0 + b;
         uint32_t t[4];
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), key.worker, key.step,
-                      key.seed_lo, key.seed_hi, t);
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), rk.worker, rk.step, rk, t);
         for (int k = 0; k < 4; ++k) y[4 * b + k] = t[k];
     }
     const unsigned shift = (unsigned)(g0 & 7u);       // first element's field in the 40-field run
@@ -78,6 +102,22 @@ static __device__ __noinline__ void draw_row_unaligned(uint64_t g0, const DrawKe
         const uint32_t hi = (y[f1 >> 1] >> (16u * (f1 & 1u))) & 0xFFFFu;
         h[j] = lo | (hi << 16);
     }
+}
+
+// max(m, |a|, |b|) in one three-input instruction.
+__device__ __forceinline__ float max3_abs(float m, float a, float b)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b)));
+    return r;
+}
+
+__device__ __forceinline__ float row_abs_max(const float (&x)[32])
+{
+    float mx = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) mx = max3_abs(mx, x[j], x[j + 1]);
+    return mx;
 }
 
 // Per-bucket encode constants, pre-scaled by 2^16: T = fma(x, inv16, half_l16) = 2^16 * t with
@@ -122,30 +162,36 @@ constexpr uint32_t kCodeBias = 0x4B400000u;      // bit pattern of 1.5 * 2^23
 __device__ __forceinline__ float draw_lo(uint32_t y) { return __uint_as_float(__byte_perm(y, 0x4B000000u, 0x7610)); }
 __device__ __forceinline__ float draw_hi(uint32_t y) { return __uint_as_float(__byte_perm(y, 0x4B000000u, 0x7632)); }
 
+// Sum (mod 2^32) of the kCodeBias contributions that land in word k of a packed row.
+template <int BITS>
+__host__ __device__ constexpr uint32_t pack_bias(int k)
+{
+    uint32_t b = 0;
+    for (int j = 0; j < 32; ++j) {
+        const int o = j * BITS, wi = o >> 5, sh = o & 31;
+        if (wi == k) b += kCodeBias << sh;
+        if (sh + BITS > 32 && wi + 1 == k) b += kCodeBias >> (32 - sh);
+    }
+    return b;
+}
+
 // Encode the 32 values of a row and pack them, code j at bits [j*BITS, j*BITS+BITS), into BITS
-// words.  The biased patterns kCodeBias + q are accumulated with multiply-adds; the bias
-// contributions are compile-time constants removed at the end.
+// words.  The biased patterns kCodeBias + q are accumulated with shift-adds; the first
+// contribution to a word also removes that word's total bias (a compile-time constant).
 template <int BITS>
 __device__ __forceinline__ void encode_pack_row(const float (&x)[32], const EncodeScale& e,
                                                 const uint32_t (&h)[16], uint32_t (&w)[BITS])
 {
-    uint32_t bias[BITS];
-#pragma unroll
-    for (int k = 0; k < BITS; ++k) { w[k] = 0u; bias[k] = 0u; }
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         const float hf = (j & 1) ? draw_hi(h[j >> 1]) : draw_lo(h[j >> 1]);
         const uint32_t c = encode_bits(x[j], e, hf);
         const int o = j * BITS, wi = o >> 5, sh = o & 31;
-        w[wi] += c << sh;
-        bias[wi] += kCodeBias << sh;
-        if (sh + BITS > 32) {
-            w[wi + 1] += c >> (32 - sh);          // the bias has 22 zero low bits: no carry mixes in
-            bias[wi + 1] += kCodeBias >> (32 - sh);
-        }
+        if (sh == 0) w[wi] = c - pack_bias<BITS>(wi);
+        else w[wi] = w[wi] + (c << sh);
+        if (sh + BITS > 32)                                     // the bias has 22 zero low bits:
+            w[wi + 1] = (c >> (32 - sh)) - pack_bias<BITS>(wi + 1);   // no carry mixes in
     }
-#pragma unroll
-    for (int k = 0; k < BITS; ++k) w[k] -= bias[k];
 }
 
 // Code j of a row from its BITS words.

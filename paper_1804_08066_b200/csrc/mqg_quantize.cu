@@ -81,9 +81,7 @@ quantize_pack_kernel(const QuantizeArgs a)
         for (int j = 0; j < 32; ++j) x[j] = 0.0f;
     }
 
-    float mx = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(x[j]));
+    const float mx = row_abs_max(x);
 
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const uint32_t mbits = bucket_max(__float_as_uint(mx), a.rows_per_bucket, local_bucket, active,
@@ -98,7 +96,7 @@ quantize_pack_kernel(const QuantizeArgs a)
     const EncodeScale es = encode_scale<BITS>(s);
     const uint64_t row = row0 + t;
     uint32_t h[16];
-    if constexpr (ALIGNED_DRAWS) draw_row_aligned(a.elem_offset + row * 32, a.key, h);
+    if constexpr (ALIGNED_DRAWS) draw_row_aligned(a.elem_offset + row * 32, make_round_keys(a.key), h);
     else draw_row_unaligned(a.elem_offset + row * 32, a.key, h);
 
     uint32_t w[BITS];
@@ -165,116 +163,155 @@ __device__ __noinline__ void stage_ragged_row(uint8_t* stage, int row, const voi
     }
 }
 
-template <int BITS, int DTYPE, int THREADS, int STAGES>
-__global__ void __launch_bounds__(THREADS)
-quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const QuantizeArgs a,
-                    unsigned int* __restrict__ timeouts)
+template <int DTYPE, int THREADS>
+struct TmaQuantizeShared {
+    static constexpr int kRowBytes = DTYPE == 0 ? 128 : 64;
+    // depth of the shared-memory ring: two stages where they fit in 32 KB, else one (the refill
+    // of a single stage still hides behind the tile's arithmetic)
+    static constexpr int kStages = 2 * THREADS * kRowBytes <= 32768 ? 2 : 1;
+    alignas(1024) uint8_t stage[kStages][THREADS * kRowBytes];
+    uint32_t slots[3][THREADS / 32];       // bucket maxima, rotating so no reset races a use
+    alignas(8) uint64_t bar[kStages];
+};
+
+// Kernel-constant inputs of the TMA kernel beyond QuantizeArgs: the ten Philox round keys are
+// computed on the host so the kernel reads them as constant operands.
+struct TmaQuantizeConsts {
+    RoundKeys rk;
+    uint32_t full_tiles;         // leading tiles whose rows are all complete and in range
+    uint32_t blk0_lo, blk0_hi;   // Philox block index of element 0: elem_offset / 8
+};
+
+// One tile, the k-th of this CTA.  FULL: every thread owns a complete row (no bounds checks).
+// SHUFFLE: a bucket is an aligned power-of-two group of at most 32 rows (lane shuffles);
+// otherwise a whole number of warps (one shared-memory atomic per warp).  After the tile's
+// rows are in registers the stage is refilled with tile `next_tile`.  Returns false if the
+// tile's copy never landed.
+template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE>
+__device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh,
+                                              const CUtensorMap* tmap, const QuantizeArgs a,
+                                              const TmaQuantizeConsts c, uint32_t k, uint32_t tile,
+                                              uint32_t next_tile, uint32_t box_bytes,
+                                              uint32_t local_bucket, bool scale_writer)
 {
-    constexpr int ROW_BYTES = DTYPE == 0 ? 128 : 64;
-    constexpr int STAGE_BYTES = THREADS * ROW_BYTES;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint32_t* slots = reinterpret_cast<uint32_t*>(base + STAGES * STAGE_BYTES);      // [3][THREADS]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(slots + 3 * THREADS);               // [STAGES]
+    constexpr int kQuantStages = TmaQuantizeShared<DTYPE, THREADS>::kStages;
+    const uint32_t t = threadIdx.x;
+    const uint32_t row = tile * a.tile_rows + t;
+    const bool active = FULL || (t < a.tile_rows && row < (uint32_t)a.nrows);
+    const uint32_t stg = k % kQuantStages, parity = (k / kQuantStages) & 1;
+    const uint32_t bar = smem_u32(&sh.bar[stg]);
+    uint8_t* stage = sh.stage[stg];
+
+    bool ok = mbar_try_wait(bar, parity);
+    if (!ok) ok = mbar_wait(bar, parity);
+
+    float x[32];
+    if (active) {
+        if (!FULL && row >= (uint32_t)a.nrows_full)
+            stage_ragged_row<DTYPE>(stage, (int)t, a.grad, (uint64_t)row * 32, a.n);
+        read_row_swizzled<DTYPE>(stage, (int)t, x);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) x[j] = 0.0f;
+    }
+    uint32_t m = __float_as_uint(row_abs_max(x));
+    uint32_t* slot = sh.slots[k % 3];
+    if (SHUFFLE) {
+        for (uint32_t d = a.rows_per_bucket >> 1; d > 0; d >>= 1)
+            m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+    } else {
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        if ((t & 31) == 0) atomicMax(&slot[local_bucket], m);
+    }
+    if (__syncthreads_or(!ok)) return false;
+    if (t == 0 && next_tile < a.ntiles) {                        // every thread has read the stage
+        mbar_expect_tx(bar, box_bytes);
+        tma_load_2d(smem_u32(stage), tmap, 0, (int)(next_tile * a.tile_rows), bar);
+    }
+    if (!SHUFFLE) {
+        m = slot[local_bucket];
+        if (t < THREADS / 32) sh.slots[(k + 2) % 3][t] = 0u;     // next used by this CTA's tile k + 2
+    }
+    if (!active) return true;
+
+    float sc = __uint_as_float(m);
+    if (sc < flush_limit()) sc = 0.0f;
+    const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
+    if (scale_writer && (FULL || bucket < a.nbuckets)) a.scales[bucket] = sc;
+
+    const EncodeScale es = encode_scale<BITS>(sc);
+    uint32_t h[16];
+    {
+        // Philox block of the row's first element: elem_offset / 8 + 4 * row (64-bit)
+        const uint32_t lo = c.blk0_lo + 4u * row;
+        const uint32_t hi = c.blk0_hi + (row >> 30) + (lo < c.blk0_lo ? 1u : 0u);
+        draw_row_blocks(lo, hi, c.rk, h);
+    }
+    uint32_t w[BITS];
+    encode_pack_row<BITS>(x, es, h, w);
+    const uint64_t word0 = (uint64_t)row * BITS;
+    if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
+        store_row_words<BITS>(a.codes, word0, w);
+    } else {
+        mask_row_words<BITS>(w, (int)(a.n - (uint64_t)row * 32) * BITS);
+#pragma unroll
+        for (int j = 0; j < BITS; ++j)
+            if (word0 + j < a.ncode_words) a.codes[word0 + j] = w[j];
+    }
+    return true;
+}
+
+template <int BITS, int DTYPE, int THREADS, bool SHUFFLE>
+__global__ void __launch_bounds__(THREADS, 768 / THREADS)
+quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ QuantizeArgs a,
+                    const __grid_constant__ TmaQuantizeConsts c, unsigned int* __restrict__ timeouts)
+{
+    using Shared = TmaQuantizeShared<DTYPE, THREADS>;
+    constexpr int kQuantStages = Shared::kStages;
+    __shared__ Shared sh;
 
     const uint32_t t = threadIdx.x;
-    const uint32_t my_count = a.ntiles > blockIdx.x ? (a.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    const uint32_t box_bytes = a.tile_rows * ROW_BYTES;
-    const uint32_t rpb = a.rows_per_bucket;
-    const bool shuffle_only = (rpb & (rpb - 1)) == 0 && rpb <= 32;
-
+    const uint32_t stride = gridDim.x;
+    const uint32_t box_bytes = a.tile_rows * Shared::kRowBytes;
     if (t == 0) {
-        for (int s = 0; s < STAGES; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        for (int s = 0; s < kQuantStages; ++s) mbar_init(smem_u32(&sh.bar[s]), 1);
         fence_barrier_init();
     }
-    for (int i = t; i < 3 * THREADS; i += THREADS) slots[i] = 0u;
+    if (t < 3 * (THREADS / 32)) (&sh.slots[0][0])[t] = 0u;
     __syncthreads();
-
-    auto issue = [&](uint32_t k) {
-        const int s = k % STAGES;
-        const uint32_t tile = blockIdx.x + k * gridDim.x;
-        const uint32_t bar = smem_u32(&bars[s]);
-        mbar_expect_tx(bar, box_bytes);
-        tma_load_2d(smem_u32(base + s * STAGE_BYTES), &tmap, 0, (int)(tile * a.tile_rows), bar);
-    };
+    uint32_t tile = blockIdx.x;
     if (t == 0) {
         prefetch_tensormap(&tmap);
-        for (uint32_t k = 0; k < (uint32_t)STAGES && k < my_count; ++k) issue(k);
+        for (uint32_t s = 0; s < (uint32_t)kQuantStages && tile + s * stride < a.ntiles; ++s) {
+            mbar_expect_tx(smem_u32(&sh.bar[s]), box_bytes);
+            tma_load_2d(smem_u32(sh.stage[s]), &tmap, 0, (int)((tile + s * stride) * a.tile_rows),
+                        smem_u32(&sh.bar[s]));
+        }
     }
+    const uint32_t local_bucket = t / a.rows_per_bucket;
+    const bool scale_writer = (t % a.rows_per_bucket) == 0;
+    const uint32_t ahead = kQuantStages * stride;       // distance to the tile that refills a stage
 
-    const uint32_t local_bucket = t / rpb;
-    const bool scale_writer = (t % rpb) == 0;
     uint32_t k = 0;
-    bool failed = false;
-    for (; k < my_count; ++k) {
-        const int s = k % STAGES;
-        const uint32_t tile = blockIdx.x + k * gridDim.x;
-        const uint64_t row0 = (uint64_t)tile * a.tile_rows;
-        const uint64_t rows_left = a.nrows - row0;
-        const uint32_t rows = rows_left < a.tile_rows ? (uint32_t)rows_left : a.tile_rows;
-        const bool active = t < rows;
-        const uint64_t row = row0 + t;
-
-        const bool ok = mbar_wait(smem_u32(&bars[s]), (k / STAGES) & 1);
-
-        float x[32];
-        if (active) {
-            if (row >= a.nrows_full)
-                stage_ragged_row<DTYPE>(base + s * STAGE_BYTES, (int)t, a.grad, row * 32, a.n);
-            read_row_swizzled<DTYPE>(base + s * STAGE_BYTES, (int)t, x);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) x[j] = 0.0f;
-        }
-        float mx = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(x[j]));
-        uint32_t m = __float_as_uint(mx);
-
-        uint32_t* slot = slots + (k % 3) * THREADS;
-        if (shuffle_only) {
-            for (uint32_t d = rpb >> 1; d > 0; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
-        } else {
-            m = __reduce_max_sync(0xFFFFFFFFu, m);        // rpb % 32 == 0: a warp is inside one bucket
-            if ((t & 31) == 0 && active) atomicMax(&slot[local_bucket], m);
-        }
-        failed = __syncthreads_or(!ok) != 0;
-        if (failed) break;
-        if (t == 0 && k + STAGES < my_count) issue(k + STAGES);      // every thread has read stage s
-        if (!shuffle_only) {
-            m = slot[local_bucket];
-            if (t < a.buckets_per_tile) slots[((k + 2) % 3) * THREADS + t] = 0u;   // next use: tile k + 2
-        }
-        if (!active) continue;
-
-        float sc = __uint_as_float(m);
-        if (sc < flush_limit()) sc = 0.0f;
-        const uint64_t bucket = (uint64_t)tile * a.buckets_per_tile + local_bucket;
-        if (scale_writer && bucket < a.nbuckets) a.scales[bucket] = sc;
-
-        const EncodeScale es = encode_scale<BITS>(sc);
-        uint32_t h[16];
-        draw_row_aligned(a.elem_offset + row * 32, a.key, h);
-        uint32_t w[BITS];
-        encode_pack_row<BITS>(x, es, h, w);
-
-        const uint64_t word0 = row * BITS;
-        if (row * 32 + 32 <= a.n) {
-            store_row_words<BITS>(a.codes, word0, w);
-        } else {
-            mask_row_words<BITS>(w, (int)(a.n - row * 32) * BITS);
-#pragma unroll
-            for (int j = 0; j < BITS; ++j)
-                if (word0 + j < a.ncode_words) a.codes[word0 + j] = w[j];
-        }
-    }
-    if (failed) {
-        // a copy never landed: record it, wait (bounded) for the copies still in flight so that
-        // none can write into shared memory after this CTA has gone, and leave
+    bool ok = true;
+#pragma unroll 1
+    for (; ok && tile < c.full_tiles; tile += stride, ++k)
+        ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, &tmap, a, c, k, tile, tile + ahead,
+                                                                 box_bytes, local_bucket, scale_writer);
+#pragma unroll 1
+    for (; ok && tile < a.ntiles; tile += stride, ++k)
+        ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, &tmap, a, c, k, tile, tile + ahead,
+                                                                  box_bytes, local_bucket, scale_writer);
+    if (!ok) {
+        // A copy never landed: record it, then give the copies still in flight (the one that was
+        // being waited for and those issued after it) a last bounded chance to finish before the
+        // CTA's shared memory can be handed to another CTA.  The loop's update ran once after the
+        // failing tile, so that tile is k - 1 / tile - stride.
         if (t == 0) {
             atomicAdd(timeouts, 1u);
-            for (uint32_t j = k; j < my_count && j < k + STAGES; ++j)
-                mbar_wait(smem_u32(&bars[j % STAGES]), (j / STAGES) & 1);
+            uint32_t j = k - 1, tl = tile - stride;
+            for (int s = 0; s < kQuantStages && tl < a.ntiles; ++s, ++j, tl += stride)
+                mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1);
         }
         __syncthreads();
     }
@@ -295,48 +332,44 @@ static cudaError_t launch_bits(const QuantizeArgs& a, int dtype, bool aligned, u
     return cudaGetLastError();
 }
 
-template <int BITS, int DTYPE, int THREADS>
-static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a, unsigned int* timeouts,
+template <int BITS, int DTYPE, int THREADS, bool SHUFFLE>
+static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a,
+                                   const TmaQuantizeConsts& c, unsigned int* timeouts,
                                    cudaStream_t stream)
 {
-    constexpr int STAGES = 3;
-    constexpr int ROW_BYTES = DTYPE == 0 ? 128 : 64;
-    constexpr size_t smem = 1024 + (size_t)STAGES * THREADS * ROW_BYTES + 3 * THREADS * 4 + STAGES * 8;
-    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, STAGES>;
-    static int ctas_per_sm[64] = {};               // per device; 0 = not yet configured
+    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, SHUFFLE>;
+    static int grid_cap[64] = {};                  // per device; 0 = not yet queried
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
-    static int sm_count[64] = {};
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (ctas_per_sm[dev] == 0) {
-        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (grid_cap[dev] == 0) {
+        int occ = 0, sms = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, THREADS, 0);
         if (err != cudaSuccess) return err;
-        int occ = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, THREADS, smem);
-        if (err != cudaSuccess) return err;
-        int sms = 0;
         err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (err != cudaSuccess) return err;
-        sm_count[dev] = sms;
-        ctas_per_sm[dev] = occ > 0 ? occ : 1;
+        grid_cap[dev] = sms * (occ > 0 ? occ : 1);
     }
-    unsigned grid = (unsigned)sm_count[dev] * (unsigned)ctas_per_sm[dev];
+    unsigned grid = (unsigned)grid_cap[dev];
     if (grid > a.ntiles) grid = a.ntiles;
-    kernel<<<grid, THREADS, smem, stream>>>(map, a, timeouts);
+    kernel<<<grid, THREADS, 0, stream>>>(map, a, c, timeouts);
     return cudaGetLastError();
 }
 
 template <int BITS>
-static cudaError_t launch_tma_bits(const CUtensorMap& map, const QuantizeArgs& a, int dtype, int threads,
+static cudaError_t launch_tma_bits(const CUtensorMap& map, const QuantizeArgs& a,
+                                   const TmaQuantizeConsts& c, int dtype, int threads, bool shuffle,
                                    unsigned int* timeouts, cudaStream_t stream)
 {
+#define MQG_TMA_CASE(D, T, S) return launch_tma_inst<BITS, D, T, S>(map, a, c, timeouts, stream)
     if (dtype == 0) {
-        if (threads == 128) return launch_tma_inst<BITS, 0, 128>(map, a, timeouts, stream);
-        return launch_tma_inst<BITS, 0, 256>(map, a, timeouts, stream);
+        if (threads == 128) { if (shuffle) MQG_TMA_CASE(0, 128, true); else MQG_TMA_CASE(0, 128, false); }
+        MQG_TMA_CASE(0, 256, false);
     }
-    if (threads == 128) return launch_tma_inst<BITS, 1, 128>(map, a, timeouts, stream);
-    return launch_tma_inst<BITS, 1, 256>(map, a, timeouts, stream);
+    if (threads == 128) { if (shuffle) MQG_TMA_CASE(1, 128, true); else MQG_TMA_CASE(1, 128, false); }
+    MQG_TMA_CASE(1, 256, false);
+#undef MQG_TMA_CASE
 }
 
 // TMA path: whole rows exist, draws are block-aligned, and a bucket is either an aligned
@@ -380,15 +413,25 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
         unsigned int* timeouts = wait_timeout_counter();
         if (timeouts != nullptr &&
             encode_rows_map(&map, grad, a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why)) {
+            TmaQuantizeConsts c;
+            uint32_t k0 = a.key.seed_lo, k1 = a.key.seed_hi;
+            for (int r = 0; r < 10; ++r) {
+                c.rk.k0[r] = k0; c.rk.k1[r] = k1;
+                k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+            }
+            c.rk.worker = worker; c.rk.step = step;
+            c.full_tiles = a.tile_rows == (uint32_t)threads ? (uint32_t)(a.nrows_full / a.tile_rows) : 0u;
+            c.blk0_lo = (uint32_t)(elem_offset >> 3); c.blk0_hi = (uint32_t)(elem_offset >> 35);
+            const bool shuffle = rpb <= 32;
             switch (bits) {
-                case 1: return launch_tma_bits<1>(map, a, dtype, threads, timeouts, stream);
-                case 2: return launch_tma_bits<2>(map, a, dtype, threads, timeouts, stream);
-                case 3: return launch_tma_bits<3>(map, a, dtype, threads, timeouts, stream);
-                case 4: return launch_tma_bits<4>(map, a, dtype, threads, timeouts, stream);
-                case 5: return launch_tma_bits<5>(map, a, dtype, threads, timeouts, stream);
-                case 6: return launch_tma_bits<6>(map, a, dtype, threads, timeouts, stream);
-                case 7: return launch_tma_bits<7>(map, a, dtype, threads, timeouts, stream);
-                case 8: return launch_tma_bits<8>(map, a, dtype, threads, timeouts, stream);
+                case 1: return launch_tma_bits<1>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 2: return launch_tma_bits<2>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 3: return launch_tma_bits<3>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 4: return launch_tma_bits<4>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 5: return launch_tma_bits<5>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 6: return launch_tma_bits<6>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 7: return launch_tma_bits<7>(map, a, c, dtype, threads, shuffle, timeouts, stream);
+                case 8: return launch_tma_bits<8>(map, a, c, dtype, threads, shuffle, timeouts, stream);
             }
             return cudaErrorInvalidValue;
         }

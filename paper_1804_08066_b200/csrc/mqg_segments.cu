@@ -93,7 +93,7 @@ encode_segments_kernel(const SegQuantArgs a, const SegmentTable tab)
     const EncodeScale es = encode_scale<BITS>(s);
     const uint64_t g0 = a.elem_offset + g.elem0 + 32ull * t;
     uint32_t h[16];
-    if ((g0 & 7u) == 0) draw_row_aligned(g0, a.key, h);
+    if ((g0 & 7u) == 0) draw_row_aligned(g0, make_round_keys(a.key), h);
     else draw_row_unaligned(g0, a.key, h);
 
     uint32_t w[BITS];

@@ -73,8 +73,11 @@ def test_quantize_shapes_and_ragged_tails(bits, n, bucket):
 
 
 @pytest.mark.parametrize("bits", [1, 3, 4, 7, 8])
-@pytest.mark.parametrize("elem_offset", [8, 4096, (1 << 35) + 64, 3, 2049, (1 << 40) + 5])
+@pytest.mark.parametrize("elem_offset", [8, 4096, (1 << 35) + 64, 3, 2049, (1 << 40) + 5,
+                                         (1 << 35) - 16, (1 << 35) - 8 * 4 * 5 - 8, (1 << 35) - 13])
 def test_quantize_elem_offset(bits, elem_offset):
+    """Offsets that are block-aligned or not, beyond 32 bits, and whose Philox block index
+    crosses 2^32 inside a row and between rows."""
     x = wl.normal(10_000, 1e-3, config=12, worker=0)
     assert_quantize_parity(x, bits, 512, seed=0xFEDCBA9876543210, worker=5, step=17,
                            elem_offset=elem_offset)
