@@ -398,12 +398,43 @@ __device__ __forceinline__ DecodeScale decode_scale(float s)
     return d;
 }
 
-// m = the float 2^23 + q (code merged into the mantissa of 2^23).
-template <int BITS>
-__device__ __forceinline__ float decode_biased(float m, const DecodeScale& d)
+// ---------------------------------------------------------------------------------
+// Packed fp32x2 arithmetic of sm_100: one instruction rounds two independent fp32 lanes, each
+// exactly as the scalar instruction with the same rounding mode would.  It halves the issue
+// slots of the decode arithmetic.
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
 {
-    constexpr float kOff = 8388608.0f + (float)(((1 << BITS) - 2) / 2);   // 2^23 + (L - 1) / 2
-    return __fmaf_rn(__fsub_rn(m, kOff), d.two_h, d.minus_h);
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t r, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ uint64_t fma2_rn(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2_rn(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// Two codes at once.  m2 = the floats 2^23 + q (code merged into the mantissa of 2^23);
+// returns v2 + x^ for both lanes, each x^ rounded once, then the sum rounded once.
+template <int BITS>
+__device__ __forceinline__ uint64_t accumulate2(uint64_t v2, uint64_t m2, uint64_t two_h2,
+                                                uint64_t minus_h2)
+{
+    constexpr float kNegOff = -(8388608.0f + (float)(((1 << BITS) - 2) / 2));   // -(2^23 + (L - 1) / 2)
+    const uint64_t qi = add2_rn(m2, pack2(kNegOff, kNegOff));                   // q - (L - 1) / 2, exact
+    return add2_rn(v2, fma2_rn(qi, two_h2, minus_h2));
 }
 
 __device__ __forceinline__ float byte_to_biased(uint32_t v, int byte)
@@ -411,53 +442,72 @@ __device__ __forceinline__ float byte_to_biased(uint32_t v, int byte)
     return __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7650 + byte));
 }
 
-// v[] <- v[] + de-quantized row, v must hold the running sum (+0 before the first worker:
-// 0 + x^ is exact, and turns the -0 of a zero-scale bucket into +0).
+// v2[] <- v2[] + de-quantized row; v2[p] holds the running sums of elements 2p and 2p+1 (+0
+// before the first worker: 0 + x^ is exact, and turns the -0 of a zero-scale bucket into +0).
 template <int BITS>
 __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const DecodeScale& d,
-                                                float (&v)[32])
+                                                uint64_t (&v2)[16])
 {
     if constexpr (BITS == 1) {
-        // x^ = +-s: flip the sign of s (= 2h - h... h itself) where the code bit is 0
+        // x^ = +-s (s = h for one bit): set the sign where the code bit is 0
         const uint32_t sbits = __float_as_uint(-d.minus_h);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const uint32_t sign = (~(w[0] << (31 - j))) & 0x80000000u;
-            v[j] = __fadd_rn(v[j], __uint_as_float(sbits | sign));
-        }
-    } else if constexpr (BITS == 8) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-            v[j] = __fadd_rn(v[j], decode_biased<8>(byte_to_biased(w[j >> 2], j & 3), d));
-    } else if constexpr (BITS == 4) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                v[8 * k + 2 * b] = __fadd_rn(v[8 * k + 2 * b], decode_biased<4>(byte_to_biased(lo, b), d));
-                v[8 * k + 2 * b + 1] = __fadd_rn(v[8 * k + 2 * b + 1], decode_biased<4>(byte_to_biased(hi, b), d));
-            }
-        }
-    } else if constexpr (BITS == 2) {
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const uint32_t t = (w[k] >> (2 * r)) & 0x03030303u;
-#pragma unroll
-                for (int b = 0; b < 4; ++b)
-                    v[16 * k + 4 * b + r] = __fadd_rn(v[16 * k + 4 * b + r],
-                                                      decode_biased<2>(byte_to_biased(t, b), d));
-            }
+        for (int p = 0; p < 16; ++p) {
+            const uint32_t s0 = (~(w[0] << (31 - 2 * p))) & 0x80000000u;
+            const uint32_t s1 = (~(w[0] << (30 - 2 * p))) & 0x80000000u;
+            v2[p] = add2_rn(v2[p], pack2(__uint_as_float(sbits | s0), __uint_as_float(sbits | s1)));
         }
     } else {
+        const uint64_t th2 = pack2(d.two_h, d.two_h), mh2 = pack2(d.minus_h, d.minus_h);
+        if constexpr (BITS == 8) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const uint32_t q = unpack_one<BITS>(w, j);
-            v[j] = __fadd_rn(v[j], decode_biased<BITS>(__uint_as_float(q | 0x4B000000u), d));
+            for (int p = 0; p < 16; ++p)
+                v2[p] = accumulate2<8>(v2[p], pack2(byte_to_biased(w[p >> 1], (2 * p) & 3),
+                                                    byte_to_biased(w[p >> 1], (2 * p + 1) & 3)), th2, mh2);
+        } else if constexpr (BITS == 4) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+                for (int b = 0; b < 4; ++b)      // elements 8k + 2b (low nibble) and 8k + 2b + 1 (high)
+                    v2[4 * k + b] = accumulate2<4>(v2[4 * k + b],
+                                                   pack2(byte_to_biased(lo, b), byte_to_biased(hi, b)), th2, mh2);
+            }
+        } else if constexpr (BITS == 2) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                uint32_t t[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) t[r] = (w[k] >> (2 * r)) & 0x03030303u;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {    // element 16k + 4b + r lives in byte b of t[r]
+                    v2[8 * k + 2 * b] = accumulate2<2>(v2[8 * k + 2 * b],
+                                                       pack2(byte_to_biased(t[0], b), byte_to_biased(t[1], b)), th2, mh2);
+                    v2[8 * k + 2 * b + 1] = accumulate2<2>(v2[8 * k + 2 * b + 1],
+                                                           pack2(byte_to_biased(t[2], b), byte_to_biased(t[3], b)), th2, mh2);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int p = 0; p < 16; ++p) {
+                const uint32_t q0 = unpack_one<BITS>(w, 2 * p), q1 = unpack_one<BITS>(w, 2 * p + 1);
+                v2[p] = accumulate2<BITS>(v2[p], pack2(__uint_as_float(q0 | 0x4B000000u),
+                                                       __uint_as_float(q1 | 0x4B000000u)), th2, mh2);
+            }
         }
     }
+}
+
+// v[] (32 floats) <-> v2[] (16 packed pairs)
+__device__ __forceinline__ void pairs_from_floats(const float (&v)[32], uint64_t (&v2)[16])
+{
+#pragma unroll
+    for (int p = 0; p < 16; ++p) v2[p] = pack2(v[2 * p], v[2 * p + 1]);
+}
+__device__ __forceinline__ void floats_from_pairs(const uint64_t (&v2)[16], float (&v)[32])
+{
+#pragma unroll
+    for (int p = 0; p < 16; ++p) unpack2(v2[p], v[2 * p], v[2 * p + 1]);
 }
 
 }  // namespace mqg

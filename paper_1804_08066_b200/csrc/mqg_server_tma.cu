@@ -3,8 +3,8 @@
 // copy into a swizzled shared-memory stage, are updated in place and leave by a tiled bulk
 // store, so parameter traffic never passes through registers of more than one thread and is
 // always full 128-byte lines.  The W code streams are read straight from global memory with
-// 128/64/32-bit loads (a thread's row is K consecutive words per worker), software-pipelined
-// one worker ahead.  Per-(worker, bucket) de-quantization constants are computed once per tile
+// 128/64/32-bit loads (a thread's row is K consecutive words per worker), a group of workers
+// at a time, the first group one tile ahead.  Per-(worker, bucket) de-quantization constants are computed once per tile
 // into a small shared table, one tile ahead.
 #include "mqg_common.cuh"
 #include "mqg_internal.h"
@@ -56,6 +56,16 @@ __device__ __forceinline__ void fill_scale_table(const ServerTmaArgs& a, float2 
     }
 }
 
+// Requests the code words of workers g0 .. g0+GROUP-1 (those that exist) for one row.
+template <int BITS, int GROUP>
+__device__ __forceinline__ void load_group(const ServerTmaArgs& a, int g0, uint64_t word0,
+                                           uint32_t (&wbuf)[GROUP][BITS])
+{
+#pragma unroll
+    for (int i = 0; i < GROUP; ++i)
+        if (g0 + i < a.W) load_row_words<BITS>(a.ptrs.codes[g0 + i], word0, wbuf[i]);
+}
+
 template <int BITS>
 __global__ void __launch_bounds__(kSrvThreads, 5)
 server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ ServerTmaArgs a,
@@ -80,6 +90,11 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         tma_load_2d(smem_u32(sh.stage[0]), &tmap, 0, (int)(tile * kSrvThreads), smem_u32(&sh.bar[0]));
     }
 
+    constexpr int kGroup = BITS <= 4 ? 8 : 32 / BITS;        // workers whose words are in flight together
+    uint32_t wbuf[kGroup][BITS];
+    if (tile < a.full_tiles)
+        load_group<BITS, kGroup>(a, 0, (uint64_t)(tile * kSrvThreads + t) * BITS, wbuf);
+
     uint32_t k = 0;
     bool failed = false;
 #pragma unroll 1
@@ -99,38 +114,44 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         const uint32_t row = tile * kSrvThreads + t;
         const uint32_t lb = bucket_of_row(a, row) - bucket_of_row(a, tile * kSrvThreads);
         const uint64_t word0 = (uint64_t)row * BITS;
-        float v[32];
+        uint64_t v2[16];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = 0.0f;
-        uint32_t cur[BITS], nxt[BITS];
-        load_row_words<BITS>(a.ptrs.codes[0], word0, cur);
+        for (int p = 0; p < 16; ++p) v2[p] = 0ull;
+        // Workers are taken in groups of kGroup whose code words are all requested before any is
+        // decoded.  The first group of this tile was requested at the end of the previous
+        // iteration (or before the loop), so its latency is already covered.
 #pragma unroll 1
-        for (int w = 0; w < a.W; ++w) {
-            if (w + 1 < a.W) load_row_words<BITS>(a.ptrs.codes[w + 1], word0, nxt);
-            const float2 e = sh.table[stg][w][lb];
-            DecodeScale d;
-            d.two_h = e.x; d.minus_h = e.y;
-            add_decoded_row<BITS>(cur, d, v);
+        for (int g0 = 0; g0 < a.W; g0 += kGroup) {
+            if (g0 > 0) load_group<BITS, kGroup>(a, g0, word0, wbuf);
 #pragma unroll
-            for (int j = 0; j < BITS; ++j) cur[j] = nxt[j];
+            for (int i = 0; i < kGroup; ++i) {
+                if (g0 + i < a.W) {
+                    const float2 e = sh.table[stg][g0 + i][lb];
+                    DecodeScale d; d.two_h = e.x; d.minus_h = e.y;
+                    add_decoded_row<BITS>(wbuf[i], d, v2);
+                }
+            }
         }
 
         bool ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
         if (!ok) ok = mbar_wait(smem_u32(&sh.bar[stg]), parity);
 
         // params <- fma(-lr, sum, params), in place in the stage
-        float4* tl = reinterpret_cast<float4*>(sh.stage[stg]);
+        {
+            uint4* tl = reinterpret_cast<uint4*>(sh.stage[stg]);
+            const uint64_t nlr2 = pack2(a.neg_lr, a.neg_lr);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const int idx = swz((int)t, c);
-            float4 p = tl[idx];
-            p.x = __fmaf_rn(a.neg_lr, v[4 * c], p.x);
-            p.y = __fmaf_rn(a.neg_lr, v[4 * c + 1], p.y);
-            p.z = __fmaf_rn(a.neg_lr, v[4 * c + 2], p.z);
-            p.w = __fmaf_rn(a.neg_lr, v[4 * c + 3], p.w);
-            tl[idx] = p;
+            for (int c = 0; c < 8; ++c) {
+                const int idx = swz((int)t, c);
+                const uint4 p = tl[idx];
+                const uint64_t lo = fma2_rn(nlr2, v2[2 * c], ((uint64_t)p.y << 32) | p.x);
+                const uint64_t hi = fma2_rn(nlr2, v2[2 * c + 1], ((uint64_t)p.w << 32) | p.z);
+                tl[idx] = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32));
+            }
         }
         fence_proxy_async();                                   // the bulk store must see these writes
+        if (tile + stride < a.full_tiles)                      // first worker group of the next tile
+            load_group<BITS, kGroup>(a, 0, (uint64_t)((tile + stride) * kSrvThreads + t) * BITS, wbuf);
         // constants of this CTA's next tile; table[stg ^ 1] was last read two barriers ago
         if (tile + stride < a.full_tiles) fill_scale_table<BITS>(a, sh.table[stg ^ 1], tile + stride);
         failed = __syncthreads_or(!ok) != 0;
@@ -158,17 +179,19 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
             const uint64_t e0 = (uint64_t)row * 32;
             const uint64_t word0 = (uint64_t)row * BITS;
             const uint32_t bucket = bucket_of_row(a, row);
-            float v[32];
+            uint64_t v2[16];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+            for (int p = 0; p < 16; ++p) v2[p] = 0ull;
             for (int w = 0; w < a.W; ++w) {
                 uint32_t cw[BITS];
 #pragma unroll
                 for (int j = 0; j < BITS; ++j)
                     cw[j] = (word0 + j < a.ncode_words) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
                 const DecodeScale d = decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket));
-                add_decoded_row<BITS>(cw, d, v);
+                add_decoded_row<BITS>(cw, d, v2);
             }
+            float v[32];
+            floats_from_pairs(v2, v);
 #pragma unroll
             for (int j = 0; j < 32; ++j)
                 if (e0 + j < a.n) a.params[e0 + j] = __fmaf_rn(a.neg_lr, v[j], a.params[e0 + j]);
