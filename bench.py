@@ -221,6 +221,21 @@ def run_reference(args):
     return 0
 
 
+def slowest_rank_ms(ms, dist, device):
+    """Elapsed time of the job = the slowest rank's (every rank runs an independent replica)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(world, grad_bytes_per_rank_step, ms_per_step):
+    """Aggregate throughput of `world` replicas that each push grad_bytes per step."""
+    return world * grad_bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
 def workload_config():
     return {"workload": "configs[1]: flat ResNet-50-sized gradient, n=25,000,000 fp32 per worker, W=8, "
                         "iid Laplace(0,1e-4), bucket 2048, bits 1..8",
@@ -316,11 +331,7 @@ def run_ours(args):
             torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return slowest_rank_ms(ms, dist, "cuda")
 
     # ---- device-resident timing
     for i in range(args.warmup):
@@ -337,7 +348,7 @@ def run_ours(args):
     total_ms = max_over_ranks(t_begin.elapsed_time(t_end))
     ms_per_step = total_ms / args.steps
     grad_bytes_per_step = len(ALL_BITS) * W * 4 * n
-    value = world * grad_bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(world, grad_bytes_per_step, ms_per_step)
 
     q_ms = {b: [] for b in ALL_BITS}
     s_ms = {b: [] for b in ALL_BITS}
@@ -382,7 +393,7 @@ def run_ours(args):
     b1.record(stream)
     barrier()
     e2e_ms = max_over_ranks(b0.elapsed_time(b1)) / e2e_steps
-    e2e = {"value": world * grad_bytes_per_step / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+    e2e = {"value": whole_job_gbs(world, grad_bytes_per_step, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": grad_bytes_per_step, "d2h_bytes_per_step": len(ALL_BITS) * 4 * n,
            "ms_per_step": e2e_ms, "steps": e2e_steps}
 

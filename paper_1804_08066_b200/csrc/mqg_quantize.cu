@@ -278,10 +278,12 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
         fence_barrier_init();
     }
     if (t < 3 * (THREADS / 32)) (&sh.slots[0][0])[t] = 0u;
+    if (t == 0) prefetch_tensormap(&tmap);
+    grid_dependency_release();
     __syncthreads();
+    grid_dependency_wait();            // nothing above touches global memory
     uint32_t tile = blockIdx.x;
     if (t == 0) {
-        prefetch_tensormap(&tmap);
         for (uint32_t s = 0; s < (uint32_t)kQuantStages && tile + s * stride < a.ntiles; ++s) {
             mbar_expect_tx(smem_u32(&sh.bar[s]), box_bytes);
             tma_load_2d(smem_u32(sh.stage[s]), &tmap, 0, (int)((tile + s * stride) * a.tile_rows),
@@ -353,8 +355,7 @@ static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a
     }
     unsigned grid = (unsigned)grid_cap[dev];
     if (grid > a.ntiles) grid = a.ntiles;
-    kernel<<<grid, THREADS, 0, stream>>>(map, a, c, timeouts);
-    return cudaGetLastError();
+    return launch_pdl(kernel, grid, THREADS, stream, map, a, c, timeouts);
 }
 
 template <int BITS>

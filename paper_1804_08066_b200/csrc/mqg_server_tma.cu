@@ -81,11 +81,13 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         mbar_init(smem_u32(&sh.bar[1]), 1);
         fence_barrier_init();
     }
+    if (t == 0) prefetch_tensormap(&tmap);
+    grid_dependency_release();
+    grid_dependency_wait();            // nothing above touches global memory
     uint32_t tile = blockIdx.x;
     if (tile < a.full_tiles) fill_scale_table<BITS>(a, sh.table[0], tile);
     __syncthreads();
     if (t == 0 && tile < a.full_tiles) {
-        prefetch_tensormap(&tmap);
         mbar_expect_tx(smem_u32(&sh.bar[0]), kTileBytes);
         tma_load_2d(smem_u32(sh.stage[0]), &tmap, 0, (int)(tile * kSrvThreads), smem_u32(&sh.bar[0]));
     }
@@ -219,8 +221,7 @@ static cudaError_t launch_server_tma_bits(const CUtensorMap& map, const ServerTm
     }
     unsigned grid = (unsigned)grid_cap[dev];
     if (grid > a.full_tiles) grid = a.full_tiles;
-    kernel<<<grid, kSrvThreads, 0, stream>>>(map, a, timeouts);
-    return cudaGetLastError();
+    return launch_pdl(kernel, grid, kSrvThreads, stream, map, a, timeouts);
 }
 
 bool server_tma_applies(uint64_t n, uint64_t bucket)

@@ -97,7 +97,33 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map)
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 
+// Programmatic dependent launch.  A kernel launched with launch_pdl() may begin while the
+// previous kernel of the stream is still draining: its CTAs become resident as the earlier
+// kernel's CTAs retire and run their set-up, then block in grid_dependency_wait() until the
+// earlier kernel has completed and its writes are visible.  Every access to global memory must
+// come after that wait.  grid_dependency_release() lets the NEXT kernel be scheduled early in
+// the same way.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- host side ------------------------------------------------------------------------
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream,
+                       Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Encodes a 2-D row-major tensor map: `rows` rows of `row_elems` elements (row_bytes =
 // 64 or 128 selects the matching swizzle), box = box_rows x row_elems.  Returns false with a
 // message if the driver entry point is missing or the encode fails.

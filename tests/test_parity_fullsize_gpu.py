@@ -1,0 +1,61 @@
+"""Parity at the benchmark's full size and launch configuration: n = 25,000,000 fp32 per
+worker, W = 8, Laplace(0, 1e-4), bucket 2048 (12,207 full buckets and one of 64 elements),
+every bit width, checked element by element against the CPU checker."""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+import paper_1804_08066_b200 as mqg
+from oracle import mqg_oracle as O
+from paper_1804_08066_b200 import workloads as wl
+from tests.gpu_util import Guarded, bits_equal, max_rel_err, to_dev
+
+pytestmark = pytest.mark.gpu
+
+N, W, B, SEED, LR = 25_000_000, 8, 2048, 2, 0.1 / 8
+_cache = {}
+
+
+def _inputs():
+    if not _cache:
+        with ThreadPoolExecutor(8) as ex:
+            _cache["host"] = list(ex.map(lambda w: wl.laplace(N, 1e-4, config=2, worker=w), range(W)))
+        _cache["dev"] = [to_dev(g) for g in _cache["host"]]
+        _cache["params"] = wl.params(N, 0.05, config=2)
+    return _cache
+
+
+@pytest.mark.parametrize("bits", list(range(1, 9)))
+def test_full_size_step(bits):
+    c = _inputs()
+    with ThreadPoolExecutor(8) as ex:
+        ref = list(ex.map(lambda w: O.quantize(c["host"][w], bits, B, SEED, worker=w, step=7), range(W)))
+    codes, scales = [], []
+    differing = 0
+    for w in range(W):
+        dc = Guarded(mqg.mqg_code_words(N, bits), torch.int32)
+        ds = Guarded(mqg.mqg_num_buckets(N, B), torch.float32)
+        mqg.mqg_quantize(c["dev"][w], N, bits, B, SEED, dc.view, ds.view, worker=w, step=7)
+        torch.cuda.synchronize()
+        dc.check_guards(), ds.check_guards()
+        assert bits_equal(ds.numpy(np.float32), ref[w][1]) == 0
+        got = dc.numpy(np.uint32)
+        if not np.array_equal(got, ref[w][0]):
+            differing += int((O.unpack(got, N, bits) != O.unpack(ref[w][0], N, bits)).sum())
+        codes.append(dc), scales.append(ds)
+    # the stated bar allows threshold ties up to 1e-6 of n; none are expected
+    assert differing <= 1e-6 * N * W
+    assert differing == 0
+    assert mqg.mqg_wire_bytes(N, bits, B) == 4 * ref[0][0].size + 4 * ref[0][1].size
+
+    p_ref, _ = O.server_step([r[0] for r in ref], [r[1] for r in ref], bits, N, B, c["params"].copy(), LR)
+    p = Guarded(N, torch.float32, fill=c["params"])
+    mqg.mqg_server_step([d.view for d in codes], [d.view for d in scales], W, bits, N, B, p.view, LR)
+    torch.cuda.synchronize()
+    p.check_guards()
+    got = p.numpy(np.float32)
+    assert max_rel_err(got, p_ref) <= 1e-6
+    assert bits_equal(got, p_ref) == 0
+    assert mqg.mqg_device_timeouts() == 0
