@@ -384,6 +384,18 @@ struct DecodeScale {
     float two_h, minus_h;
 };
 
+// The same constants duplicated for the two lanes of the packed instructions.
+struct DecodeScale2 {
+    float2 two_h, minus_h;
+};
+__device__ __forceinline__ DecodeScale2 widen(const DecodeScale& d)
+{
+    DecodeScale2 r;
+    r.two_h = make_float2(d.two_h, d.two_h);
+    r.minus_h = make_float2(d.minus_h, d.minus_h);
+    return r;
+}
+
 template <int BITS>
 __device__ __forceinline__ DecodeScale decode_scale(float s)
 {
@@ -399,71 +411,51 @@ __device__ __forceinline__ DecodeScale decode_scale(float s)
 }
 
 // ---------------------------------------------------------------------------------
-// Packed fp32x2 arithmetic of sm_100: one instruction rounds two independent fp32 lanes, each
-// exactly as the scalar instruction with the same rounding mode would.  It halves the issue
-// slots of the decode arithmetic.
+// Packed fp32x2 arithmetic of sm_100 (__fadd2_rn, __ffma2_rn on float2): one instruction rounds
+// two independent fp32 lanes, each exactly as the scalar instruction would.  It halves the
+// issue slots of the decode arithmetic.
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t pack2(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t r, float& lo, float& hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
-}
-__device__ __forceinline__ uint64_t fma2_rn(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2_rn(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 
-// Two codes at once.  m2 = the floats 2^23 + q (code merged into the mantissa of 2^23);
-// returns v2 + x^ for both lanes, each x^ rounded once, then the sum rounded once.
+// Two codes at once.  m = the floats 2^23 + q (code merged into the mantissa of 2^23);
+// returns v + x^ for both lanes, each x^ rounded once, then the sum rounded once.
 template <int BITS>
-__device__ __forceinline__ uint64_t accumulate2(uint64_t v2, uint64_t m2, uint64_t two_h2,
-                                                uint64_t minus_h2)
+__device__ __forceinline__ float2 accumulate2(float2 v, float2 m, float2 two_h, float2 minus_h)
 {
     constexpr float kNegOff = -(8388608.0f + (float)(((1 << BITS) - 2) / 2));   // -(2^23 + (L - 1) / 2)
-    const uint64_t qi = add2_rn(m2, pack2(kNegOff, kNegOff));                   // q - (L - 1) / 2, exact
-    return add2_rn(v2, fma2_rn(qi, two_h2, minus_h2));
+    const float2 qi = __fadd2_rn(m, make_float2(kNegOff, kNegOff));             // q - (L - 1) / 2, exact
+    return __fadd2_rn(v, __ffma2_rn(qi, two_h, minus_h));
 }
 
-__device__ __forceinline__ float byte_to_biased(uint32_t v, int byte)
+// `bias` is the bit pattern of 2^23 (0x4B000000).  Callers pass it from a kernel argument so that
+// it is a constant-bank operand of the byte permute instead of a register that has to be
+// re-materialised when registers are short.
+__device__ __forceinline__ float byte_to_biased(uint32_t v, int byte, uint32_t bias)
 {
-    return __uint_as_float(__byte_perm(v, 0x4B000000u, 0x7650 + byte));
+    return __uint_as_float(__byte_perm(v, bias, 0x7650 + byte));
 }
 
 // v2[] <- v2[] + de-quantized row; v2[p] holds the running sums of elements 2p and 2p+1 (+0
 // before the first worker: 0 + x^ is exact, and turns the -0 of a zero-scale bucket into +0).
 template <int BITS>
-__device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const DecodeScale& d,
-                                                uint64_t (&v2)[16])
+__device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const DecodeScale2& d,
+                                                float2 (&v2)[16], uint32_t bias = 0x4B000000u)
 {
     if constexpr (BITS == 1) {
         // x^ = +-s (s = h for one bit): set the sign where the code bit is 0
-        const uint32_t sbits = __float_as_uint(-d.minus_h);
+        const uint32_t sbits = __float_as_uint(-d.minus_h.x);
 #pragma unroll
         for (int p = 0; p < 16; ++p) {
             const uint32_t s0 = (~(w[0] << (31 - 2 * p))) & 0x80000000u;
             const uint32_t s1 = (~(w[0] << (30 - 2 * p))) & 0x80000000u;
-            v2[p] = add2_rn(v2[p], pack2(__uint_as_float(sbits | s0), __uint_as_float(sbits | s1)));
+            v2[p] = __fadd2_rn(v2[p], make_float2(__uint_as_float(sbits | s0), __uint_as_float(sbits | s1)));
         }
     } else {
-        const uint64_t th2 = pack2(d.two_h, d.two_h), mh2 = pack2(d.minus_h, d.minus_h);
+        const float2 th = d.two_h, mh = d.minus_h;
         if constexpr (BITS == 8) {
 #pragma unroll
             for (int p = 0; p < 16; ++p)
-                v2[p] = accumulate2<8>(v2[p], pack2(byte_to_biased(w[p >> 1], (2 * p) & 3),
-                                                    byte_to_biased(w[p >> 1], (2 * p + 1) & 3)), th2, mh2);
+                v2[p] = accumulate2<8>(v2[p], make_float2(byte_to_biased(w[p >> 1], (2 * p) & 3, bias),
+                                                          byte_to_biased(w[p >> 1], (2 * p + 1) & 3, bias)), th, mh);
         } else if constexpr (BITS == 4) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -471,7 +463,7 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
 #pragma unroll
                 for (int b = 0; b < 4; ++b)      // elements 8k + 2b (low nibble) and 8k + 2b + 1 (high)
                     v2[4 * k + b] = accumulate2<4>(v2[4 * k + b],
-                                                   pack2(byte_to_biased(lo, b), byte_to_biased(hi, b)), th2, mh2);
+                                                   make_float2(byte_to_biased(lo, b, bias), byte_to_biased(hi, b, bias)), th, mh);
             }
         } else if constexpr (BITS == 2) {
 #pragma unroll
@@ -482,32 +474,32 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {    // element 16k + 4b + r lives in byte b of t[r]
                     v2[8 * k + 2 * b] = accumulate2<2>(v2[8 * k + 2 * b],
-                                                       pack2(byte_to_biased(t[0], b), byte_to_biased(t[1], b)), th2, mh2);
+                                                       make_float2(byte_to_biased(t[0], b, bias), byte_to_biased(t[1], b, bias)), th, mh);
                     v2[8 * k + 2 * b + 1] = accumulate2<2>(v2[8 * k + 2 * b + 1],
-                                                           pack2(byte_to_biased(t[2], b), byte_to_biased(t[3], b)), th2, mh2);
+                                                           make_float2(byte_to_biased(t[2], b, bias), byte_to_biased(t[3], b, bias)), th, mh);
                 }
             }
         } else {
 #pragma unroll
             for (int p = 0; p < 16; ++p) {
                 const uint32_t q0 = unpack_one<BITS>(w, 2 * p), q1 = unpack_one<BITS>(w, 2 * p + 1);
-                v2[p] = accumulate2<BITS>(v2[p], pack2(__uint_as_float(q0 | 0x4B000000u),
-                                                       __uint_as_float(q1 | 0x4B000000u)), th2, mh2);
+                v2[p] = accumulate2<BITS>(v2[p], make_float2(__uint_as_float(q0 | bias),
+                                                             __uint_as_float(q1 | bias)), th, mh);
             }
         }
     }
 }
 
-// v[] (32 floats) <-> v2[] (16 packed pairs)
-__device__ __forceinline__ void pairs_from_floats(const float (&v)[32], uint64_t (&v2)[16])
+// v[] (32 floats) <-> v2[] (16 pairs)
+__device__ __forceinline__ void pairs_from_floats(const float (&v)[32], float2 (&v2)[16])
 {
 #pragma unroll
-    for (int p = 0; p < 16; ++p) v2[p] = pack2(v[2 * p], v[2 * p + 1]);
+    for (int p = 0; p < 16; ++p) v2[p] = make_float2(v[2 * p], v[2 * p + 1]);
 }
-__device__ __forceinline__ void floats_from_pairs(const uint64_t (&v2)[16], float (&v)[32])
+__device__ __forceinline__ void floats_from_pairs(const float2 (&v2)[16], float (&v)[32])
 {
 #pragma unroll
-    for (int p = 0; p < 16; ++p) unpack2(v2[p], v[2 * p], v[2 * p + 1]);
+    for (int p = 0; p < 16; ++p) { v[2 * p] = v2[p].x; v[2 * p + 1] = v2[p].y; }
 }
 
 }  // namespace mqg

@@ -29,11 +29,11 @@ __device__ __forceinline__ void accumulate_row(const ServerArgs& a, uint64_t sca
                                                uint64_t word0, uint64_t words_end, bool full_row,
                                                float (&v)[32], bool have_init)
 {
-    uint64_t v2[16];
+    float2 v2[16];
     if (have_init) pairs_from_floats(v, v2);
     else {
 #pragma unroll
-        for (int p = 0; p < 16; ++p) v2[p] = 0ull;
+        for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
     }
     for (int wk = 0; wk < a.W; ++wk) {
         uint32_t w[BITS];
@@ -43,7 +43,7 @@ __device__ __forceinline__ void accumulate_row(const ServerArgs& a, uint64_t sca
             for (int k = 0; k < BITS; ++k)
                 w[k] = (word0 + k < words_end) ? __ldg(a.ptrs.codes[wk] + word0 + k) : 0u;
         }
-        const DecodeScale d = decode_scale<BITS>(__ldg(a.ptrs.scales[wk] + scale_idx));
+        const DecodeScale2 d = widen(decode_scale<BITS>(__ldg(a.ptrs.scales[wk] + scale_idx)));
         add_decoded_row<BITS>(w, d, v2);
     }
     floats_from_pairs(v2, v);

@@ -13,7 +13,7 @@
 namespace mqg {
 
 constexpr int kSrvThreads = 128;        // rows per tile = threads per CTA
-constexpr int kSrvMaxBuckets = 18;      // buckets one tile can touch when a bucket has >= 8 rows
+constexpr int kSrvMaxBuckets = 10;      // buckets one tile can touch when a bucket has >= 16 rows
 
 struct ServerTmaArgs {
     WorkerPtrs ptrs;
@@ -26,11 +26,12 @@ struct ServerTmaArgs {
     int rpb_shift;               // log2(rows_per_bucket) if a power of two, else -1
     int W;
     float neg_lr;
+    uint32_t bias_bits;          // 0x4B000000 (2^23), a run-time constant for the byte permutes
 };
 
 struct ServerTmaShared {
     alignas(1024) uint8_t stage[2][kSrvThreads * 128];
-    float2 table[2][kMaxWorkers][kSrvMaxBuckets];     // (2h, -h) per worker and bucket of the tile
+    float4 table[2][kMaxWorkers][kSrvMaxBuckets];     // (2h, 2h, -h, -h) per worker and bucket of the tile
     alignas(8) uint64_t bar[2];
 };
 
@@ -41,7 +42,7 @@ __device__ __forceinline__ uint32_t bucket_of_row(const ServerTmaArgs& a, uint32
 
 // De-quantization constants of every (worker, bucket) pair the tile touches.
 template <int BITS>
-__device__ __forceinline__ void fill_scale_table(const ServerTmaArgs& a, float2 (*table)[kSrvMaxBuckets],
+__device__ __forceinline__ void fill_scale_table(const ServerTmaArgs& a, float4 (*table)[kSrvMaxBuckets],
                                                  uint32_t tile)
 {
     const uint32_t first = bucket_of_row(a, tile * kSrvThreads);
@@ -52,7 +53,7 @@ __device__ __forceinline__ void fill_scale_table(const ServerTmaArgs& a, float2 
         float s = 0.0f;
         if (first + lb < a.nbuckets) s = __ldg(a.ptrs.scales[w] + first + lb);
         const DecodeScale d = decode_scale<BITS>(s);
-        table[w][lb] = make_float2(d.two_h, d.minus_h);
+        table[w][lb] = make_float4(d.two_h, d.two_h, d.minus_h, d.minus_h);
     }
 }
 
@@ -116,9 +117,9 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
         const uint32_t row = tile * kSrvThreads + t;
         const uint32_t lb = bucket_of_row(a, row) - bucket_of_row(a, tile * kSrvThreads);
         const uint64_t word0 = (uint64_t)row * BITS;
-        uint64_t v2[16];
+        float2 v2[16];
 #pragma unroll
-        for (int p = 0; p < 16; ++p) v2[p] = 0ull;
+        for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
         // Workers are taken in groups of kGroup whose code words are all requested before any is
         // decoded.  The first group of this tile was requested at the end of the previous
         // iteration (or before the loop), so its latency is already covered.
@@ -128,9 +129,10 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
 #pragma unroll
             for (int i = 0; i < kGroup; ++i) {
                 if (g0 + i < a.W) {
-                    const float2 e = sh.table[stg][g0 + i][lb];
-                    DecodeScale d; d.two_h = e.x; d.minus_h = e.y;
-                    add_decoded_row<BITS>(wbuf[i], d, v2);
+                    const float4 e = sh.table[stg][g0 + i][lb];
+                    DecodeScale2 d;
+                    d.two_h = make_float2(e.x, e.y); d.minus_h = make_float2(e.z, e.w);
+                    add_decoded_row<BITS>(wbuf[i], d, v2, a.bias_bits);
                 }
             }
         }
@@ -140,15 +142,15 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
 
         // params <- fma(-lr, sum, params), in place in the stage
         {
-            uint4* tl = reinterpret_cast<uint4*>(sh.stage[stg]);
-            const uint64_t nlr2 = pack2(a.neg_lr, a.neg_lr);
+            float4* tl = reinterpret_cast<float4*>(sh.stage[stg]);
+            const float2 nlr = make_float2(a.neg_lr, a.neg_lr);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int idx = swz((int)t, c);
-                const uint4 p = tl[idx];
-                const uint64_t lo = fma2_rn(nlr2, v2[2 * c], ((uint64_t)p.y << 32) | p.x);
-                const uint64_t hi = fma2_rn(nlr2, v2[2 * c + 1], ((uint64_t)p.w << 32) | p.z);
-                tl[idx] = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32));
+                const float4 p = tl[idx];
+                const float2 lo = __ffma2_rn(nlr, v2[2 * c], make_float2(p.x, p.y));
+                const float2 hi = __ffma2_rn(nlr, v2[2 * c + 1], make_float2(p.z, p.w));
+                tl[idx] = make_float4(lo.x, lo.y, hi.x, hi.y);
             }
         }
         fence_proxy_async();                                   // the bulk store must see these writes
@@ -181,15 +183,15 @@ server_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constan
             const uint64_t e0 = (uint64_t)row * 32;
             const uint64_t word0 = (uint64_t)row * BITS;
             const uint32_t bucket = bucket_of_row(a, row);
-            uint64_t v2[16];
+            float2 v2[16];
 #pragma unroll
-            for (int p = 0; p < 16; ++p) v2[p] = 0ull;
+            for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
             for (int w = 0; w < a.W; ++w) {
                 uint32_t cw[BITS];
 #pragma unroll
                 for (int j = 0; j < BITS; ++j)
                     cw[j] = (word0 + j < a.ncode_words) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
-                const DecodeScale d = decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket));
+                const DecodeScale2 d = widen(decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
                 add_decoded_row<BITS>(cw, d, v2);
             }
             float v[32];
@@ -228,7 +230,7 @@ bool server_tma_applies(uint64_t n, uint64_t bucket)
 {
     const uint64_t nrows = (n + 31) / 32;
     const uint64_t rpb = bucket >= n ? nrows : bucket / 32;
-    return n / 32 >= (uint64_t)kSrvThreads && nrows <= 0x7FFFFFFFull && rpb >= 8;
+    return n / 32 >= (uint64_t)kSrvThreads && nrows <= 0x7FFFFFFFull && rpb >= 16;
 }
 
 cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
@@ -249,6 +251,7 @@ cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
         if (((uint64_t)1 << sft) == rpb) a.rpb_shift = sft;
     a.W = W;
     a.neg_lr = -lr;
+    a.bias_bits = 0x4B000000u;
     CUtensorMap map;
     const char* why = nullptr;
     unsigned int* timeouts = wait_timeout_counter();
