@@ -52,7 +52,7 @@ cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, 
 cudaError_t launch_server(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                           float* params, float lr, float* acc, int add_into, cudaStream_t stream);
 
-// TMA-fed fused server pass (params update, no acc output, uniform buckets of >= 16 rows).
+// TMA-fed fused server pass (params update, no acc output, uniform buckets of >= 32 rows).
 bool server_tma_applies(uint64_t n, uint64_t bucket);
 cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                               float* params, float lr, cudaStream_t stream);
