@@ -84,8 +84,13 @@ __device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float4
     }
 }
 
+// CTAs per SM the register budget is set for: the decode of the wider codes schedules better
+// with up to 128 registers (4 CTAs = 16 warps per SM) than with 5 CTAs and 102 registers.
 template <int BITS>
-__global__ void __launch_bounds__(kSrvThreads, 5)
+constexpr int server_min_ctas() { return BITS == 1 ? 5 : 4; }
+
+template <int BITS>
+__global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
 server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ CUtensorMap map_tail,
                   const __grid_constant__ ServerTmaArgs a, unsigned int* __restrict__ timeouts)
 {
