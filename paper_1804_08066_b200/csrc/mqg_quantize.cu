@@ -262,7 +262,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
 }
 
 template <int BITS, int DTYPE, int THREADS, bool SHUFFLE>
-__global__ void __launch_bounds__(THREADS, 640 / THREADS)
+__global__ void __launch_bounds__(THREADS, 512 / THREADS)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ QuantizeArgs a,
                     const __grid_constant__ TmaQuantizeConsts c, unsigned int* __restrict__ timeouts)
 {
