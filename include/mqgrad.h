@@ -112,6 +112,21 @@ mqg_status mqg_server_step(const uint32_t* const* codes, const float* const* sca
                            void* cuda_stream);
 
 /*
+ * The server's downlink (ReceiveQGThenSendQG of Algorithm 1, lines 3-5; steps 6-8 of Fig. 3): the
+ * global gradient g = (sum_p g_p) * mean_scale, with the sum as in mqg_dequant_accumulate and one
+ * rounding for the product (pass mean_scale = 1 / P for the paper's mean), is quantized again with
+ * the same bit width and bucket, exactly as mqg_quantize(g, ...) with elem_offset 0 would, without
+ * storing g.  Workers then apply it with mqg_server_step(W = 1, lr = eta).
+ *   codes_out, scales_out [out] laid out as mqg_quantize writes them
+ *   worker, step               key the random draws of this encode (use an id no worker uses)
+ * Buckets (or a single bucket n) above 8192 elements are rejected with MQG_ERR_INVALID.
+ */
+mqg_status mqg_server_requantize(const uint32_t* const* codes, const float* const* scales, int W,
+                                 int bits, uint64_t n, uint64_t bucket, float mean_scale,
+                                 uint64_t seed, uint32_t* codes_out, float* scales_out,
+                                 uint32_t worker, uint32_t step, void* cuda_stream);
+
+/*
  * Per-layer scale ("gradient quantization is applied to these two layers", Section 4.1): the flat
  * gradient is cut into nseg segments; segment j = elements [seg_off[j], seg_off[j+1]) is ONE bucket
  * with scale scales[j], and its bit stream starts on a word boundary at word code_off[j].

@@ -240,6 +240,25 @@ int mqo_server_step(const uint32_t *const *codes, const float *const *scales, in
     return rc;
 }
 
+/* Downlink of the server (ReceiveQGThenSendQG, lines 3-5): the mean of the de-quantized worker
+ * gradients, g = (sum_p g_p) * mean_scale with one rounding for the product, is quantized again
+ * with the same K and bucket size (elem_offset 0) for the broadcast. */
+int mqo_server_requantize(const uint32_t *const *codes, const float *const *scales, int W, int bits,
+                          uint64_t n, uint64_t bucket, float mean_scale, uint64_t seed,
+                          uint32_t *codes_out, float *scales_out, uint32_t worker, uint32_t step)
+{
+    if (n == 0) return 0;
+    float *g = (float *)malloc(n * sizeof(float));
+    if (!g) return -2;
+    int rc = mqo_dequant_accumulate(codes, scales, W, bits, n, g, bucket, 0);
+    if (rc == 0) {
+        for (uint64_t i = 0; i < n; ++i) g[i] = g[i] * mean_scale;
+        rc = mqo_quantize(g, n, bits, bucket, seed, codes_out, scales_out, 0, worker, step, 0);
+    }
+    free(g);
+    return rc;
+}
+
 /* Per-layer scale: segment j covers elements [seg_off[j], seg_off[j+1]) of the
  * flat gradient, is one bucket, and its bit stream starts at word code_off[j].
  * Element i of segment j draws with g = elem_offset + seg_off[j] + i. */

@@ -41,6 +41,8 @@ _quantize = _decl("mqo_quantize", _int, _vp, _u64, _int, _u64, _u64, _vp, _vp, _
                   _u32, _u64)
 _deq_acc = _decl("mqo_dequant_accumulate", _int, _vp, _vp, _int, _int, _u64, _vp, _u64, _int)
 _server = _decl("mqo_server_step", _int, _vp, _vp, _int, _int, _u64, _u64, _vp, C.c_float, _vp)
+_requant = _decl("mqo_server_requantize", _int, _vp, _vp, _int, _int, _u64, _u64, C.c_float, _u64, _vp, _vp,
+                _u32, _u32)
 _qseg = _decl("mqo_quantize_segments", _int, _vp, _int, _vp, _vp, _int, _u64, _vp, _vp, _int,
               _u32, _u32, _u64)
 _sseg = _decl("mqo_server_step_segments", _int, _vp, _vp, _int, _int, _int, _vp, _vp, _vp,
@@ -173,6 +175,18 @@ def server_step(codes, scales, bits, n, bucket, params, lr, want_acc=False):
     if rc:
         raise ValueError("mqo_server_step failed: %d" % rc)
     return params, acc
+
+
+def server_requantize(codes, scales, bits, n, bucket, mean_scale, seed, worker=0, step=0):
+    W = len(codes)
+    codes, ctab = _ptr_array(codes, np.uint32)
+    scales, stab = _ptr_array(scales, np.float32)
+    out_c = np.zeros(code_words(n, bits), np.uint32)
+    out_s = np.zeros(num_buckets(n, bucket) if n else 0, np.float32)
+    rc = _requant(ctab, stab, W, bits, n, bucket, mean_scale, seed, _ptr(out_c), _ptr(out_s), worker, step)
+    if rc:
+        raise ValueError("mqo_server_requantize failed: %d" % rc)
+    return out_c, out_s
 
 
 def quantize_segments(grad, seg_off, code_off, bits, seed, worker=0, step=0, elem_offset=0,

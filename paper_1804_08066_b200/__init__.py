@@ -7,7 +7,7 @@ raises.
 
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
-  mqg_quantize_segments, mqg_server_step_segments, mqg_code_words, mqg_num_buckets,
+  mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
 from __future__ import annotations
@@ -52,6 +52,7 @@ def _load() -> C.CDLL:
         "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
         "mqg_apply": (i32, [vp, vp, f32, u64, vp]),
         "mqg_server_step": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
+        "mqg_server_requantize": (i32, [vp, vp, i32, i32, u64, u64, f32, u64, vp, vp, u32, u32, vp]),
         "mqg_quantize_segments": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_server_step_segments": (i32, [vp, vp, i32, i32, i32, vp, vp, vp, f32, vp, vp]),
     }
@@ -157,6 +158,16 @@ def mqg_server_step(codes, scales, W: int, bits: int, n: int, bucket: int, param
                                 n, bucket, _dev_ptr(params, "params") if n else None, lr,
                                 _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
                                 _stream()))
+
+
+def mqg_server_requantize(codes, scales, W: int, bits: int, n: int, bucket: int, mean_scale: float,
+                          seed: int, codes_out, scales_out, worker: int = 0, step: int = 0) -> None:
+    """Downlink: de-quantize + sum + scale to the mean + quantize again, in one pass."""
+    _check(_lib.mqg_server_requantize(_ptr_table(codes, "codes"), _ptr_table(scales, "scales"), W, bits,
+                                      n, bucket, mean_scale, seed & 0xFFFFFFFFFFFFFFFF,
+                                      _dev_ptr(codes_out, "codes_out") if n else None,
+                                      _dev_ptr(scales_out, "scales_out") if n else None,
+                                      worker, step, _stream()))
 
 
 def mqg_quantize_segments(grad, seg_off, code_off, bits: int, seed: int, codes, scales,

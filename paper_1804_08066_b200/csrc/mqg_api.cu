@@ -208,6 +208,30 @@ mqg_status mqg_server_step(const uint32_t* const* codes, const float* const* sca
     return MQG_OK;
 }
 
+mqg_status mqg_server_requantize(const uint32_t* const* codes, const float* const* scales, int W,
+                                 int bits, uint64_t n, uint64_t bucket, float mean_scale,
+                                 uint64_t seed, uint32_t* codes_out, float* scales_out,
+                                 uint32_t worker, uint32_t step, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    mqg::WorkerPtrs ptrs;
+    if (mqg_status st = check_workers(codes, scales, W, n == 0, &ptrs)) return st;
+    if (n == 0) return MQG_OK;
+    const uint64_t eff = bucket < n ? bucket : n;
+    if (eff > (uint64_t)mqg::kMaxFusedBucket)
+        return fail(MQG_ERR_INVALID, "mqg_server_requantize supports buckets of at most %d elements",
+                    mqg::kMaxFusedBucket);
+    if (!codes_out || !scales_out) return fail(MQG_ERR_INVALID, "codes_out or scales_out is null");
+    if (!aligned16(codes_out)) return fail(MQG_ERR_ALIGN, "codes_out not 16-byte aligned");
+    if (!aligned4(scales_out)) return fail(MQG_ERR_ALIGN, "scales_out not 4-byte aligned");
+    const cudaError_t err = mqg::launch_requantize(ptrs, W, bits, n, bucket, mean_scale, seed, codes_out,
+                                                   scales_out, worker, step,
+                                                   static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_server_requantize", err);
+    return MQG_OK;
+}
+
 mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg_off,
                                  const uint64_t* code_off, int bits, uint64_t seed,
                                  uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,

@@ -61,6 +61,11 @@ cudaError_t launch_server_segments(const WorkerPtrs& ptrs, int W, int bits, cons
                                    int scale_base, float* params, float lr, float* acc,
                                    cudaStream_t stream);
 
+// Server downlink: de-quantize + sum + scale to the mean + quantize again (buckets <= 8192).
+cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                              float mean_scale, uint64_t seed, uint32_t* codes_out, float* scales_out,
+                              uint32_t worker, uint32_t step, cudaStream_t stream);
+
 cudaError_t launch_apply(float* params, const float* acc, float lr, uint64_t n, cudaStream_t stream);
 
 }  // namespace mqg

@@ -37,6 +37,7 @@ MUTANTS = [
     ("flush_threshold", "ldexpf(1.0f, -96)", "ldexpf(1.0f, -90)"),
     ("bf16_low_half", "(uint32_t)in[i] << 16", "(uint32_t)in[i]"),
     ("sum_skips_last_worker", "for (int w = 0; w < W; ++w) {\n        mqo_unpack", "for (int w = 0; w < W - (W > 2); ++w) {\n        mqo_unpack"),
+    ("requantize_skips_mean", "g[i] = g[i] * mean_scale;", "g[i] = g[i];"),
     ("zero_bucket_minus_zero", "if (s == 0.0f) { xhat[i] = 0.0f; continue; }", "if (s == 0.0f) { xhat[i] = -0.0f; continue; }"),
 ]
 

@@ -469,3 +469,28 @@ def test_segments_are_buckets_with_word_aligned_streams():
                 O.server_step([codes[int(coff[j]):]] * 2, [sc[j:j + 1]] * 2, bits, s, s,
                               p2[lo:lo + s], 0.25)
         assert np.array_equal(p, p2)
+
+
+# ---------------------------------------------------------------- downlink re-quantization
+@pytest.mark.parametrize("bits", [1, 2, 5, 8])
+def test_requantize_is_mean_then_quantize_and_fixes_grid_points(bits):
+    L = (1 << bits) - 1
+    n, B, W = 3000, 512, 4
+    rng = np.random.default_rng(60 + bits)
+    xs = [(rng.standard_normal(n) * 1e-3).astype(np.float32) for _ in range(W)]
+    enc = [O.quantize(x, bits, B, 11, worker=w) for w, x in enumerate(xs)]
+    codes, scales = [e[0] for e in enc], [e[1] for e in enc]
+    c2, s2 = O.server_requantize(codes, scales, bits, n, B, 0.25, seed=11, worker=99, step=4)
+    mean = (O.dequant_accumulate(codes, scales, bits, n, B).astype(np.float64) * 0.25).astype(np.float32)
+    want_c, want_s = O.quantize(mean, bits, B, 11, worker=99, step=4)
+    assert np.array_equal(c2, want_c) and np.array_equal(s2, want_s)
+    assert np.array_equal(s2, O.bucket_scales(mean, B))
+    # one worker whose scale is L * 2^e decodes onto its own grid: re-quantizing the "mean" of
+    # that single worker returns its codes and scale, whatever the draws
+    q0 = rng.integers(0, L + 1, 512, dtype=np.uint8)
+    q0[0], q0[1] = L, 0
+    sc = np.array([L * 2.0 ** -9], np.float32)
+    c1 = O.pack(q0, bits)
+    for seed in (0, 5):
+        c3, s3 = O.server_requantize([c1], [sc], bits, 512, 512, 1.0, seed=seed, worker=7)
+        assert np.array_equal(c3, c1) and s3[0] == sc[0]

@@ -292,3 +292,38 @@ def test_segments_more_than_one_launch_chunk():
     codes.check_guards(), scales.check_guards()
     assert bits_equal(scales.numpy(np.float32), s_ref) == 0
     assert np.array_equal(codes.numpy(np.uint32), c_ref)     # streams are back to back here
+
+
+# ------------------------------------------------------------------ downlink: server re-quantization
+@pytest.mark.parametrize("bits", ALL_BITS)
+@pytest.mark.parametrize("n,bucket,W", [(40, 64, 1), (8192 + 5, 2048, 3), (100_003, 4096, 4), (9000, 96, 2),
+                                        (5000, 10_000 - 1808, 5), (65_536 + 31, 512, 8)])
+def test_server_requantize(bits, n, bucket, W):
+    xs = [wl.normal(n, 2e-3, config=41, worker=w) for w in range(W)]
+    if n >= bucket:
+        for x in xs:
+            x[:bucket] = 0.0                            # a bucket whose mean is exactly zero
+    codes, scales = oracle_workers(xs, bits, bucket, seed=bits)
+    c_ref, s_ref = O.server_requantize(codes, scales, bits, n, bucket, 1.0 / W, seed=bits, worker=1000, step=3)
+    out_c = Guarded(mqg.mqg_code_words(n, bits), torch.int32)
+    out_s = Guarded(mqg.mqg_num_buckets(n, bucket), torch.float32)
+    mqg.mqg_server_requantize([to_dev(c.view(np.int32)) for c in codes], [to_dev(s) for s in scales], W, bits,
+                              n, bucket, 1.0 / W, bits, out_c.view, out_s.view, worker=1000, step=3)
+    torch.cuda.synchronize()
+    out_c.check_guards(), out_s.check_guards()
+    assert bits_equal(out_s.numpy(np.float32), s_ref) == 0
+    assert np.array_equal(out_c.numpy(np.uint32), c_ref)
+    # the worker side of the downlink: de-quantize the broadcast and update (W = 1)
+    p0 = wl.params(n, 0.05, config=41)
+    p_ref, _ = O.server_step([c_ref], [s_ref], bits, n, bucket, p0.copy(), 0.1)
+    p = Guarded(n, torch.float32, fill=p0)
+    mqg.mqg_server_step([out_c.view], [out_s.view], 1, bits, n, bucket, p.view, 0.1)
+    torch.cuda.synchronize()
+    p.check_guards()
+    assert bits_equal(p.numpy(np.float32), p_ref) == 0
+
+
+def test_server_requantize_rejects_large_buckets():
+    e = torch.zeros(16, dtype=torch.int32, device="cuda")
+    with pytest.raises(mqg.MqgError):
+        mqg.mqg_server_requantize([e], [e.view(torch.float32)], 1, 4, 100_000, 16384, 1.0, 0, e, e.view(torch.float32))
