@@ -163,11 +163,10 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         float2 v2[16];
 #pragma unroll
         for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
-#pragma unroll 1
-        for (int g0 = 0; g0 < a.W; g0 += kGroup) {
-            if (g0 > 0) load_group<BITS, kGroup>(a, g0, word0, wbuf);
+        const uint64_t word0_next = (uint64_t)min(row0 + kSrvTileRows + lane, last_row) * BITS;
+        auto decode_slots = [&](int g0, int lo, int hi) {
 #pragma unroll
-            for (int i = 0; i < kGroup; ++i) {
+            for (int i = lo; i < hi; ++i) {
                 if (g0 + i < a.W) {
                     const float4 e = sh.table[stg][g0 + i][lb];
                     DecodeScale2 d;
@@ -175,6 +174,28 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
                     add_decoded_row<BITS>(wbuf[i], d, v2, a.bias_bits);
                 }
             }
+        };
+        auto prefetch_slots = [&](int lo, int hi) {      // next tile's first group into freed slots
+#pragma unroll
+            for (int i = lo; i < hi; ++i)
+                if (i < a.W) load_row_words<BITS>(a.ptrs.codes[i], word0_next, wbuf[i]);
+        };
+        constexpr int kHalf = kGroup / 2;
+        if (BITS >= 5 && a.W <= kGroup) {
+            // one group of wide codes: the slots of each half are refilled for the next tile as
+            // soon as the half has been decoded, so the requests have the rest of the tile's work
+            // to land (measured: faster for K >= 5, slower for the narrow loads of K <= 3)
+            decode_slots(0, 0, kHalf);
+            if (have_next) prefetch_slots(0, kHalf);
+            decode_slots(0, kHalf, kGroup);
+            if (have_next) prefetch_slots(kHalf, kGroup);
+        } else {
+#pragma unroll 1
+            for (int g0 = 0; g0 < a.W; g0 += kGroup) {
+                if (g0 > 0) load_group<BITS, kGroup>(a, g0, word0, wbuf);
+                decode_slots(g0, 0, kGroup);
+            }
+            if (have_next) prefetch_slots(0, kGroup);
         }
 
         bool ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
@@ -196,10 +217,8 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         }
         fence_proxy_async();                                   // the bulk store must see these writes
         if (have_next) {
-            // constants and first worker group of the next tile; table[stg ^ 1] was last read in
-            // the previous iteration
+            // constants of the next tile; table[stg ^ 1] was last read in the previous iteration
             store_tile_scales<BITS>(a, sh.table[stg ^ 1], lane, s_next);
-            load_group<BITS, kGroup>(a, 0, (uint64_t)min(row0 + kSrvTileRows + lane, last_row) * BITS, wbuf);
         }
         __syncwarp();
         if (lane == 0) {
