@@ -48,6 +48,9 @@ METRIC = "quantize+pack and dequant+accumulate+update GB/s (fp32 grad) per bit w
 UNIT = "GB/s of fp32 gradient through quantize+pack -> unpack+accumulate+update"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per element of quantize_tma_kernel<4> (ncu, n = 33,554,432):
+# (134.25 MB + 7.6 MB) / 33,554,432; writes are partly still in L2 when the kernel ends
+QUANTIZE_DRAM_BYTES_PER_ELEM_K4 = 141.85e6 / 33_554_432
 
 
 def measured_hbm_peak():
@@ -376,7 +379,10 @@ def run_ours(args):
     s_achieved = s_bytes_total / s_time_total / 1e9
     roofline = {"kernel": "quantize_pack_kernel (all bit widths, %d launches per step)" % (len(ALL_BITS) * W),
                 "bound": "hbm", "achieved": q_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
-                "unit": "GB/s", "frac": q_achieved / peak, "traffic": None,
+                "unit": "GB/s", "frac": q_achieved / peak, "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n,
+                "traffic_note": "dram read+write bytes of one K=4 launch from the ncu capture in "
+                                "profiles/quantize_tma_kernel_b4_n32M.md (n=33.5M), scaled to n=25M; "
+                                "algorithmic bytes of that launch: %d" % quantize_bytes(n, 4, B),
                 "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
     roofline_server = {"kernel": "server_kernel (fused, all bit widths, %d launches per step)" % len(ALL_BITS),
                        "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
