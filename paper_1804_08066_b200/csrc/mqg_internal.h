@@ -52,10 +52,11 @@ cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, 
 cudaError_t launch_server(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                           float* params, float lr, float* acc, int add_into, cudaStream_t stream);
 
-// TMA-fed fused server pass (params update, no acc output, uniform buckets of >= 32 rows).
+// TMA-fed server pass over uniform buckets of >= 32 rows.  mode 1: dst = params, updated with lr;
+// mode 0: dst = acc, overwritten with the sum; mode 2: dst = acc, the sum continues from it.
 bool server_tma_applies(uint64_t n, uint64_t bucket);
 cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
-                              float* params, float lr, cudaStream_t stream);
+                              float* dst, float lr, int mode, cudaStream_t stream);
 
 cudaError_t launch_server_segments(const WorkerPtrs& ptrs, int W, int bits, const SegmentTable& tab,
                                    int scale_base, float* params, float lr, float* acc,

@@ -169,8 +169,12 @@ static cudaError_t dispatch_bits(int bits, const ServerArgs& a, const SegmentTab
 cudaError_t launch_server(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                           float* params, float lr, float* acc, int add_into, cudaStream_t stream)
 {
-    if (params != nullptr && acc == nullptr && server_tma_applies(n, bucket))
-        return launch_server_tma(ptrs, W, bits, n, bucket, params, lr, stream);
+    if (server_tma_applies(n, bucket)) {
+        if (params != nullptr && acc == nullptr)
+            return launch_server_tma(ptrs, W, bits, n, bucket, params, lr, 1, stream);
+        if (params == nullptr)
+            return launch_server_tma(ptrs, W, bits, n, bucket, acc, 0.0f, add_into ? 2 : 0, stream);
+    }
     ServerArgs a;
     a.ptrs = ptrs;
     a.params = params; a.acc = acc;

@@ -89,7 +89,9 @@ __device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float4
 template <int BITS>
 constexpr int server_min_ctas() { return BITS == 1 ? 5 : 4; }
 
-template <int BITS>
+// MODE 1: dst = params, dst <- fma(-lr, sum, dst).  MODE 0: dst = acc, dst <- sum.
+// MODE 2: dst = acc, the sum continues from the value already there.
+template <int BITS, int MODE>
 __global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
 server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ CUtensorMap map_tail,
                   const __grid_constant__ ServerTmaArgs a, unsigned int* __restrict__ timeouts)
@@ -126,7 +128,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         load_tile_scales(a, r_begin, lane, s0);
         store_tile_scales<BITS>(a, sh.table[0], lane, s0);
         load_group<BITS, kGroup>(a, 0, (uint64_t)min(r_begin + lane, last_row) * BITS, wbuf);
-        if (lane == 0) {
+        if (MODE != 0 && lane == 0) {
             mbar_expect_tx(smem_u32(&sh.bar[0]), kSrvTileBytes);
             tma_load_2d(smem_u32(sh.stage[0]), &map_full, 0, (int)r_begin, smem_u32(&sh.bar[0]));
         }
@@ -140,7 +142,12 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         const bool have_next = k + 1 < ntiles;
         // The other stage held tile k-1, whose store was committed at the end of the last
         // iteration: once that store has read its source the stage can take tile k+1.
-        if (lane == 0 && have_next) {
+        if (MODE == 0) {
+            // nothing is loaded: the stage is only written by this warp, once the store that used
+            // it two tiles ago has read it
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+        } else if (lane == 0 && have_next) {
             bulk_wait_read<0>();
             const uint32_t bar = smem_u32(&sh.bar[stg ^ 1]);
             const uint32_t next0 = row0 + kSrvTileRows;
@@ -161,8 +168,22 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         const uint32_t lb = bucket_of_row(a, row) - bucket_of_row(a, row0);
         const uint64_t word0 = (uint64_t)row * BITS;
         float2 v2[16];
+        bool ok = true;
+        if constexpr (MODE == 2) {
+            // the sum continues from the accumulator: its tile is needed before the first worker
+            ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
+            if (!ok) ok = mbar_wait(smem_u32(&sh.bar[stg]), parity);
+            const float4* tl = reinterpret_cast<const float4*>(sh.stage[stg]);
 #pragma unroll
-        for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
+            for (int c = 0; c < 8; ++c) {
+                const float4 p = tl[swz((int)lane, c)];
+                v2[2 * c] = make_float2(p.x, p.y);
+                v2[2 * c + 1] = make_float2(p.z, p.w);
+            }
+        } else {
+#pragma unroll
+            for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
+        }
         const uint64_t word0_next = (uint64_t)min(row0 + kSrvTileRows + lane, last_row) * BITS;
         auto decode_slots = [&](int g0, int lo, int hi) {
 #pragma unroll
@@ -198,20 +219,24 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
             if (have_next) prefetch_slots(0, kGroup);
         }
 
-        bool ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
-        if (!ok) ok = mbar_wait(smem_u32(&sh.bar[stg]), parity);
-        if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
+        if constexpr (MODE == 1) {
+            ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
+            if (!ok) ok = mbar_wait(smem_u32(&sh.bar[stg]), parity);
+        }
+        if (MODE != 0 && !__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
 
-        // params <- fma(-lr, sum, params), in place in the stage
         {
             float4* tl = reinterpret_cast<float4*>(sh.stage[stg]);
             const float2 nlr = make_float2(a.neg_lr, a.neg_lr);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int idx = swz((int)lane, c);
-                const float4 p = tl[idx];
-                const float2 lo = __ffma2_rn(nlr, v2[2 * c], make_float2(p.x, p.y));
-                const float2 hi = __ffma2_rn(nlr, v2[2 * c + 1], make_float2(p.z, p.w));
+                float2 lo = v2[2 * c], hi = v2[2 * c + 1];
+                if constexpr (MODE == 1) {          // params <- fma(-lr, sum, params), in place
+                    const float4 p = tl[idx];
+                    lo = __ffma2_rn(nlr, lo, make_float2(p.x, p.y));
+                    hi = __ffma2_rn(nlr, hi, make_float2(p.z, p.w));
+                }
                 tl[idx] = make_float4(lo.x, lo.y, hi.x, hi.y);
             }
         }
@@ -252,7 +277,13 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         const uint32_t bucket = bucket_of_row(a, row);
         float2 v2[16];
 #pragma unroll
-        for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
+        for (int p = 0; p < 16; ++p) {
+            v2[p] = make_float2(0.0f, 0.0f);
+            if constexpr (MODE == 2) {
+                if (e0 + 2 * p < a.n) v2[p].x = a.params[e0 + 2 * p];
+                if (e0 + 2 * p + 1 < a.n) v2[p].y = a.params[e0 + 2 * p + 1];
+            }
+        }
         for (int w = 0; w < a.W; ++w) {
             uint32_t cw[BITS];
 #pragma unroll
@@ -265,15 +296,15 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         floats_from_pairs(v2, v);
 #pragma unroll
         for (int j = 0; j < 32; ++j)
-            if (e0 + j < a.n) a.params[e0 + j] = __fmaf_rn(a.neg_lr, v[j], a.params[e0 + j]);
+            if (e0 + j < a.n) a.params[e0 + j] = MODE == 1 ? __fmaf_rn(a.neg_lr, v[j], a.params[e0 + j]) : v[j];
     }
 }
 
-template <int BITS>
-static cudaError_t launch_server_tma_bits(const void* params, ServerTmaArgs& a, unsigned int* timeouts,
+template <int BITS, int MODE>
+static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, unsigned int* timeouts,
                                           cudaStream_t stream)
 {
-    auto kernel = server_tma_kernel<BITS>;
+    auto kernel = server_tma_kernel<BITS, MODE>;
     static int grid_cap[64] = {};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -304,6 +335,15 @@ static cudaError_t launch_server_tma_bits(const void* params, ServerTmaArgs& a, 
     return launch_pdl(kernel, (unsigned)grid, kSrvThreads, stream, map_full, map_tail, a, timeouts);
 }
 
+template <int BITS>
+static cudaError_t launch_server_tma_bits(const void* dst, ServerTmaArgs& a, int mode, unsigned int* timeouts,
+                                          cudaStream_t stream)
+{
+    if (mode == 1) return launch_server_tma_inst<BITS, 1>(dst, a, timeouts, stream);
+    if (mode == 2) return launch_server_tma_inst<BITS, 2>(dst, a, timeouts, stream);
+    return launch_server_tma_inst<BITS, 0>(dst, a, timeouts, stream);
+}
+
 bool server_tma_applies(uint64_t n, uint64_t bucket)
 {
     const uint64_t nrows = (n + 31) / 32;
@@ -311,8 +351,9 @@ bool server_tma_applies(uint64_t n, uint64_t bucket)
     return n / 32 >= 4 * (uint64_t)kSrvTileRows && nrows <= 0x7FFFFFFFull && rpb >= (uint64_t)kSrvTileRows;
 }
 
+// mode 1: dst = params (update with lr); mode 0: dst = acc (overwrite); mode 2: dst = acc (add into)
 cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
-                              float* params, float lr, cudaStream_t stream)
+                              float* params, float lr, int mode, cudaStream_t stream)
 {
     ServerTmaArgs a;
     a.ptrs = ptrs;
@@ -334,14 +375,14 @@ cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
     unsigned int* timeouts = wait_timeout_counter();
     if (timeouts == nullptr) return cudaErrorNotSupported;
     switch (bits) {
-        case 1: return launch_server_tma_bits<1>(params, a, timeouts, stream);
-        case 2: return launch_server_tma_bits<2>(params, a, timeouts, stream);
-        case 3: return launch_server_tma_bits<3>(params, a, timeouts, stream);
-        case 4: return launch_server_tma_bits<4>(params, a, timeouts, stream);
-        case 5: return launch_server_tma_bits<5>(params, a, timeouts, stream);
-        case 6: return launch_server_tma_bits<6>(params, a, timeouts, stream);
-        case 7: return launch_server_tma_bits<7>(params, a, timeouts, stream);
-        case 8: return launch_server_tma_bits<8>(params, a, timeouts, stream);
+        case 1: return launch_server_tma_bits<1>(params, a, mode, timeouts, stream);
+        case 2: return launch_server_tma_bits<2>(params, a, mode, timeouts, stream);
+        case 3: return launch_server_tma_bits<3>(params, a, mode, timeouts, stream);
+        case 4: return launch_server_tma_bits<4>(params, a, mode, timeouts, stream);
+        case 5: return launch_server_tma_bits<5>(params, a, mode, timeouts, stream);
+        case 6: return launch_server_tma_bits<6>(params, a, mode, timeouts, stream);
+        case 7: return launch_server_tma_bits<7>(params, a, mode, timeouts, stream);
+        case 8: return launch_server_tma_bits<8>(params, a, mode, timeouts, stream);
     }
     return cudaErrorInvalidValue;
 }

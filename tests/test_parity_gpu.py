@@ -187,9 +187,10 @@ def test_server_step_shapes(bits, n, bucket, W):
     assert bits_equal(p2, p_ref) == 0
 
 
-@pytest.mark.parametrize("bits", [1, 3, 6, 8])
-def test_dequant_accumulate_then_apply_equals_fused(bits):
-    n, W, B = 50_000 + 9, 4, 512
+@pytest.mark.parametrize("bits", [1, 3, 4, 6, 8])
+@pytest.mark.parametrize("n,B", [(50_000 + 9, 512), (300_000 + 9, 2048), (8 * 4096 * 33, 4096), (70_000, 1 << 20)])
+def test_dequant_accumulate_then_apply_equals_fused(bits, n, B):
+    W = 4
     xs = [wl.laplace(n, 1e-4, config=22, worker=w) for w in range(W)]
     codes, scales = oracle_workers(xs, bits, B, seed=3)
     dc = [to_dev(c.view(np.int32)) for c in codes]
