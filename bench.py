@@ -377,14 +377,14 @@ def run_ours(args):
         })
     q_achieved = q_bytes_total / q_time_total / 1e9
     s_achieved = s_bytes_total / s_time_total / 1e9
-    roofline = {"kernel": "quantize_pack_kernel (all bit widths, %d launches per step)" % (len(ALL_BITS) * W),
+    roofline = {"kernel": "quantize_tma_kernel (all bit widths, %d launches per step)" % (len(ALL_BITS) * W),
                 "bound": "hbm", "achieved": q_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
                 "unit": "GB/s", "frac": q_achieved / peak, "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n,
                 "traffic_note": "dram read+write bytes of one K=4 launch from the ncu capture in "
                                 "profiles/quantize_tma_kernel_b4_n32M.md (n=33.5M), scaled to n=25M; "
                                 "algorithmic bytes of that launch: %d" % quantize_bytes(n, 4, B),
                 "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
-    roofline_server = {"kernel": "server_kernel (fused, all bit widths, %d launches per step)" % len(ALL_BITS),
+    roofline_server = {"kernel": "server_tma_kernel (fused step, all bit widths, %d launches per step)" % len(ALL_BITS),
                        "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
                        "unit": "GB/s", "frac": s_achieved / peak, "traffic": None}
 
