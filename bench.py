@@ -291,10 +291,20 @@ def run_ours(args):
         if rc != 0:
             raise RuntimeError("libmqgrad: %d %s" % (rc, mqg.mqg_last_error()))
 
-    def quantize_all(b, step_no):
+    grad_tab = (C.c_void_p * W)(*[t.data_ptr() for t in grads])
+    batched = args.quantize_launch == "batched"
+
+    def quantize_per_worker(b, step_no):
         for w in range(W):
             check(lib.mqg_quantize(grads[w].data_ptr(), n, b, B, PHILOX_SEED, codes[b][w].data_ptr(),
                                    scales[b][w].data_ptr(), 0, w, step_no, 0, sptr))
+
+    def quantize_batched(b, step_no):
+        check(lib.mqg_quantize_workers(grad_tab, W, n, b, B, PHILOX_SEED, code_tab[b], scale_tab[b], 0, 0,
+                                       step_no, 0, sptr))
+
+    quantize_all = quantize_batched if batched else quantize_per_worker
+    q_launches = 1 if batched else W       # quantize launches per bit width
 
     def server(b):
         check(lib.mqg_server_step(code_tab[b], scale_tab[b], W, b, n, B, params[b].data_ptr(), LR,
@@ -353,6 +363,24 @@ def run_ours(args):
     grad_bytes_per_step = len(ALL_BITS) * W * 4 * n
     value = whole_job_gbs(world, grad_bytes_per_step, ms_per_step)
 
+    # the other way of launching the quantize phase, timed on its own for comparison
+    other = quantize_per_worker if batched else quantize_batched
+    other_ms = {}
+    for b in ALL_BITS:
+        for i in range(3):
+            other(b, i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            other(b, 3 + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        other_ms[b] = e0.elapsed_time(e1) / args.steps
+    if batched:                            # leave the codes as the timed path writes them
+        for b in ALL_BITS:
+            quantize_all(b, args.warmup + args.steps - 1)
+        torch.cuda.synchronize()
+
     q_ms = {b: [] for b in ALL_BITS}
     s_ms = {b: [] for b in ALL_BITS}
     for kind, b, e0, e1 in events:
@@ -362,7 +390,7 @@ def run_ours(args):
     q_bytes_total = q_time_total = 0.0
     s_bytes_total = s_time_total = 0.0
     for b in ALL_BITS:
-        tq = float(np.mean(q_ms[b])) / W * 1e-3            # per quantize launch
+        tq = float(np.mean(q_ms[b])) / W * 1e-3            # per worker's gradient
         ts = float(np.mean(s_ms[b])) * 1e-3
         qb, sb = quantize_bytes(n, b, B), server_bytes(n, b, B, W)
         q_bytes_total += qb * W; q_time_total += tq * W
@@ -374,15 +402,21 @@ def run_ours(args):
             "server_us": ts * 1e6, "server_grad_gbs": 4 * n * W / ts / 1e9, "server_moved_gbs": sb / ts / 1e9,
             "server_frac_of_measured": sb / ts / 1e9 / peak, "server_frac_of_8tbs": sb / ts / 1e9 / NOMINAL_HBM_GBS,
             "wire_bytes_per_worker": mqg.mqg_wire_bytes(n, b, B),
+            ("quantize_us_per_worker_launches" if batched else "quantize_us_one_launch"): other_ms[b] / W * 1e3,
         })
     q_achieved = q_bytes_total / q_time_total / 1e9
     s_achieved = s_bytes_total / s_time_total / 1e9
-    roofline = {"kernel": "quantize_tma_kernel (all bit widths, %d launches per step)" % (len(ALL_BITS) * W),
+    q_kernel = "quantize_workers_kernel" if batched else "quantize_tma_kernel"
+    q_per_launch = W if batched else 1     # gradients one launch encodes
+    roofline = {"kernel": "%s (all bit widths, %d launches per step, %d gradient(s) of n per launch)"
+                          % (q_kernel, len(ALL_BITS) * q_launches, q_per_launch),
                 "bound": "hbm", "achieved": q_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
-                "unit": "GB/s", "frac": q_achieved / peak, "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n,
-                "traffic_note": "dram read+write bytes of one K=4 launch from the ncu capture in "
-                                "profiles/quantize_tma_kernel_b4_n32M.md (n=33.5M), scaled to n=25M; "
-                                "algorithmic bytes of that launch: %d" % quantize_bytes(n, 4, B),
+                "unit": "GB/s", "frac": q_achieved / peak,
+                "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n * q_per_launch,
+                "traffic_note": "dram read+write bytes per element of a K=4 launch from the ncu capture in "
+                                "profiles/quantize_tma_kernel_b4_n32M.md (n=33.5M; the batched kernel runs the "
+                                "same tile code), scaled to the elements of one launch; algorithmic bytes of "
+                                "that launch: %d" % (quantize_bytes(n, 4, B) * q_per_launch),
                 "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
     roofline_server = {"kernel": "server_tma_kernel (fused step, all bit widths, %d launches per step)" % len(ALL_BITS),
                        "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
@@ -412,8 +446,9 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(), "clocks": clocks.summary(), "e2e": e2e,
-            "gpu_launches": args.steps * len(ALL_BITS) * (W + 1),
+            "config": dict(workload_config(), quantize_launch=args.quantize_launch),
+            "clocks": clocks.summary(), "e2e": e2e,
+            "gpu_launches": args.steps * len(ALL_BITS) * (q_launches + 1),
             "roofline": roofline, "roofline_server": roofline_server, "per_bits": per_bits,
         }
         if cpu is not None:
@@ -426,7 +461,7 @@ def run_ours(args):
 
 def run_single_kernel(args):
     """A few launches of one kernel on a small case (inputs still larger than L2), for profiler
-    captures and quick timing: python bench.py --kernel quantize|server --bits B [--n N]."""
+    captures and quick timing: python bench.py --kernel quantize|quantize_workers|server --bits B [--n N]."""
     import torch
 
     import paper_1804_08066_b200 as mqg
@@ -443,6 +478,18 @@ def run_single_kernel(args):
         launch = lambda i: mqg.mqg_quantize(grads[i % rot], n, b, B, PHILOX_SEED, codes[i % rot],
                                             scales[i % rot], worker=i % rot, step=i)
         nbytes = quantize_bytes(n, b, B)
+    elif args.kernel == "quantize_workers":
+        # W gradients of n elements per launch; two buffer sets, each far larger than L2
+        rot = 2
+        grads = [[torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w + W * r)).cuda()
+                  for w in range(W)] for r in range(rot)]
+        codes = [[torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(W)]
+                 for _ in range(rot)]
+        scales = [[torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(W)]
+                  for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize_workers(grads[i % rot], W, n, b, B, PHILOX_SEED, codes[i % rot],
+                                                    scales[i % rot], first_worker=0, step=i)
+        nbytes = W * quantize_bytes(n, b, B)
     else:
         g = torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=0)).cuda()
         codes = [[torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(W)]
@@ -481,7 +528,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", choices=["quantize", "server"], default=None,
+    ap.add_argument("--quantize-launch", choices=["batched", "per-worker"], default="batched",
+                    help="the step's quantize phase: one mqg_quantize_workers launch per bit width for all "
+                         "workers' gradients, or one mqg_quantize launch per worker")
+    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server"], default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--n", type=int, default=1 << 25)

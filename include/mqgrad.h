@@ -82,6 +82,23 @@ mqg_status mqg_quantize(const void* grad, uint64_t n, int bits, uint64_t bucket,
                         void* cuda_stream);
 
 /*
+ * Quantize(g_p, K) of Algorithm 1 for W workers whose gradients live on this device (P workers
+ * simulated on one GPU, or several replicas per device), in one launch where the shape allows:
+ * exactly mqg_quantize(grads[w], ..., codes[w], scales[w], worker = first_worker + w, ...) for
+ * w = 0..W-1, bit for bit, without paying the per-launch fixed cost W times.
+ *   grads, codes, scales  HOST arrays of W device pointers (read during the call only); each
+ *                         buffer as in mqg_quantize; the outputs are what mqg_server_step and
+ *                         mqg_dequant_accumulate take as codes[] / scales[]
+ * Shapes outside the one-launch kernel (buckets above 4096 elements, fewer than 2048 elements,
+ * elem_offset not a multiple of 8, W = 1) run as W launches inside the call.
+ * Errors: as mqg_quantize, per worker; MQG_ERR_TOO_MANY_WORKERS for W outside 1..MQG_MAX_WORKERS.
+ */
+mqg_status mqg_quantize_workers(const void* const* grads, int W, uint64_t n, int bits, uint64_t bucket,
+                                uint64_t seed, uint32_t* const* codes, float* const* scales,
+                                mqg_dtype dtype, uint32_t first_worker, uint32_t step,
+                                uint64_t elem_offset, void* cuda_stream);
+
+/*
  * De-quantize + sum of Algorithm 1 (ReceiveQGThenSendQG, before the division by P):
  *   acc[i] = ((x^_0[i] + x^_1[i]) + ... ) in worker order 0..W-1, fp32,
  *   x^_w[i] = (2 q - L) * (s / L) with one rounding for s / L and one for the product;

@@ -49,6 +49,7 @@ def _load() -> C.CDLL:
         "mqg_version": (i32, []),
         "mqg_device_timeouts": (i32, [C.POINTER(C.c_uint)]),
         "mqg_quantize": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
+        "mqg_quantize_workers": (i32, [vp, i32, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
         "mqg_apply": (i32, [vp, vp, f32, u64, vp]),
         "mqg_server_step": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
@@ -138,6 +139,20 @@ def mqg_quantize(grad, n: int, bits: int, bucket: int, seed: int, codes, scales,
                              _dev_ptr(codes, "codes") if n else None,
                              _dev_ptr(scales, "scales") if n else None,
                              _grad_dtype(grad), worker, step, elem_offset, _stream()))
+
+
+def mqg_quantize_workers(grads, W: int, n: int, bits: int, bucket: int, seed: int, codes, scales,
+                         first_worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    """Quantize(g_p, K) for W workers' gradients (lists of W tensors) in one launch."""
+    if len(grads) != W or len(codes) != W or len(scales) != W:
+        raise ValueError("grads, codes and scales must each hold W tensors")
+    dtypes = {_grad_dtype(g) for g in grads}
+    if len(dtypes) != 1:
+        raise TypeError("all gradients must have the same dtype")
+    _check(_lib.mqg_quantize_workers(_ptr_table(grads, "grads"), W, n, bits, bucket,
+                                     seed & 0xFFFFFFFFFFFFFFFF, _ptr_table(codes, "codes"),
+                                     _ptr_table(scales, "scales"), dtypes.pop(), first_worker, step,
+                                     elem_offset, _stream()))
 
 
 def mqg_dequant_accumulate(codes, scales, W: int, bits: int, n: int, acc, bucket: int,

@@ -64,17 +64,24 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 // four Philox blocks, block index g >> 3; element g takes half (g & 1) of word (g & 7) >> 1.
 // h[j] holds the two draws of elements 2j (low half) and 2j+1 (high half).
 // (blk_lo, blk_hi) = 64-bit block index of the row's first element.
-__device__ __forceinline__ void draw_row_blocks(uint32_t blk_lo, uint32_t blk_hi, const RoundKeys& rk,
-                                                uint32_t (&h)[16])
+// `worker` is passed beside the keys so one set of round keys can serve several workers.
+__device__ __forceinline__ void draw_row_blocks(uint32_t blk_lo, uint32_t blk_hi, uint32_t worker,
+                                                const RoundKeys& rk, uint32_t (&h)[16])
 {
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
         uint32_t y[4];
         const uint32_t lo = blk_lo + b;
-        philox4x32_10(lo, blk_hi + (lo < blk_lo ? 1u : 0u), rk.worker, rk.step, rk, y);
+        philox4x32_10(lo, blk_hi + (lo < blk_lo ? 1u : 0u), worker, rk.step, rk, y);
 #pragma unroll
         for (int k = 0; k < 4; ++k) h[4 * b + k] = y[k];
     }
+}
+
+__device__ __forceinline__ void draw_row_blocks(uint32_t blk_lo, uint32_t blk_hi, const RoundKeys& rk,
+                                                uint32_t (&h)[16])
+{
+    draw_row_blocks(blk_lo, blk_hi, rk.worker, rk, h);
 }
 
 __device__ __forceinline__ void draw_row_aligned(uint64_t g0, const RoundKeys& rk, uint32_t (&h)[16])

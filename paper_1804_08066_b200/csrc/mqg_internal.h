@@ -34,6 +34,14 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
                                   uint32_t worker, uint32_t step, uint64_t elem_offset,
                                   cudaStream_t stream);
 
+// One launch for W >= 2 workers' gradients of the same shape (host arrays of device pointers);
+// worker w draws as worker id first_worker + w.  Only when quantize_workers_applies() holds.
+bool quantize_workers_applies(int W, uint64_t n, uint64_t bucket, uint64_t elem_offset);
+cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n, int bits,
+                                    uint64_t bucket, uint64_t seed, uint32_t* const* codes,
+                                    float* const* scales, int dtype, uint32_t first_worker,
+                                    uint32_t step, uint64_t elem_offset, cudaStream_t stream);
+
 // Two-pass quantize of segments.  scales_base points at the scale of the table's first segment.
 cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, int bits,
                                      uint64_t seed, uint32_t* codes, float* scales_base, int dtype,

@@ -7,6 +7,8 @@
 // takes part in the bucket's max reduction, draws its 32 sixteen-bit random numbers from
 // four Philox blocks, encodes, packs into K words and stores them.  The gradient is read
 // from HBM exactly once.
+#include <string.h>
+
 #include "mqg_common.cuh"
 #include "mqg_internal.h"
 #include "mqg_tma.cuh"
@@ -182,16 +184,26 @@ struct TmaQuantizeConsts {
     uint32_t blk0_lo, blk0_hi;   // Philox block index of element 0: elem_offset / 8
 };
 
-// One tile, the k-th of this CTA.  FULL: every thread owns a complete row (no bounds checks).
-// SHUFFLE: a bucket is an aligned power-of-two group of at most 32 rows (lane shuffles);
-// otherwise a whole number of warps (one shared-memory atomic per warp).  After the tile's
-// rows are in registers the stage is refilled with tile `next_tile`.  Returns false if the
-// tile's copy never landed.
-template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE>
-__device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh,
-                                              const CUtensorMap* tmap, const QuantizeArgs a,
-                                              const TmaQuantizeConsts c, uint32_t k, uint32_t tile,
-                                              uint32_t next_tile, uint32_t box_bytes,
+// What a tile needs to know about the worker it belongs to.  The one-worker kernel builds it
+// from its kernel parameters (so every member stays a constant operand), the batched kernel from
+// its table.
+struct WorkerView {
+    const CUtensorMap* map;
+    const void* grad;
+    uint32_t* codes;
+    float* scales;
+    uint32_t worker;             // third counter word of the draws
+};
+
+// One tile, the k-th of this CTA, tile `tile` of worker `wv`.  FULL: every thread owns a complete
+// row (no bounds checks).  SHUFFLE: a bucket is an aligned power-of-two group of at most 32 rows
+// (lane shuffles); otherwise a whole number of warps (one shared-memory atomic per warp).  After
+// the tile's rows are in registers thread 0 calls `refill(stage, bar)` to start the copy that
+// uses the stage next.  Returns false if the tile's copy never landed.
+template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, typename Refill>
+__device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
+                                              const QuantizeArgs& a, const TmaQuantizeConsts& c,
+                                              uint32_t k, uint32_t tile, Refill&& refill,
                                               uint32_t local_bucket, bool scale_writer)
 {
     constexpr int kQuantStages = TmaQuantizeShared<DTYPE, THREADS>::kStages;
@@ -208,7 +220,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     float x[32];
     if (active) {
         if (!FULL && row >= (uint32_t)a.nrows_full)
-            stage_ragged_row<DTYPE>(stage, (int)t, a.grad, (uint64_t)row * 32, a.n);
+            stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
         read_row_swizzled<DTYPE>(stage, (int)t, x);
     } else {
 #pragma unroll
@@ -224,10 +236,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
         if ((t & 31) == 0) atomicMax(&slot[local_bucket], m);
     }
     if (__syncthreads_or(!ok)) return false;
-    if (t == 0 && next_tile < a.ntiles) {                        // every thread has read the stage
-        mbar_expect_tx(bar, box_bytes);
-        tma_load_2d(smem_u32(stage), tmap, 0, (int)(next_tile * a.tile_rows), bar);
-    }
+    if (t == 0) refill(smem_u32(stage), bar);                    // every thread has read the stage
     if (!SHUFFLE) {
         m = slot[local_bucket];
         if (t < THREADS / 32) sh.slots[(k + 2) % 3][t] = 0u;     // next used by this CTA's tile k + 2
@@ -237,7 +246,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     float sc = __uint_as_float(m);
     if (sc < flush_limit()) sc = 0.0f;
     const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
-    if (scale_writer && (FULL || bucket < a.nbuckets)) a.scales[bucket] = sc;
+    if (scale_writer && (FULL || bucket < a.nbuckets)) wv.scales[bucket] = sc;
 
     const EncodeScale es = encode_scale<BITS>(sc);
     uint32_t h[16];
@@ -245,18 +254,18 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
         // Philox block of the row's first element: elem_offset / 8 + 4 * row (64-bit)
         const uint32_t lo = c.blk0_lo + 4u * row;
         const uint32_t hi = c.blk0_hi + (row >> 30) + (lo < c.blk0_lo ? 1u : 0u);
-        draw_row_blocks(lo, hi, c.rk, h);
+        draw_row_blocks(lo, hi, wv.worker, c.rk, h);
     }
     uint32_t w[BITS];
     encode_pack_row<BITS>(x, es, h, w);
     const uint64_t word0 = (uint64_t)row * BITS;
     if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
-        store_row_words<BITS>(a.codes, word0, w);
+        store_row_words<BITS>(wv.codes, word0, w);
     } else {
         mask_row_words<BITS>(w, (int)(a.n - (uint64_t)row * 32) * BITS);
 #pragma unroll
         for (int j = 0; j < BITS; ++j)
-            if (word0 + j < a.ncode_words) a.codes[word0 + j] = w[j];
+            if (word0 + j < a.ncode_words) wv.codes[word0 + j] = w[j];
     }
     return true;
 }
@@ -293,17 +302,26 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const bool scale_writer = (t % a.rows_per_bucket) == 0;
     const uint32_t ahead = kQuantStages * stride;       // distance to the tile that refills a stage
+    const WorkerView wv = {&tmap, a.grad, a.codes, a.scales, c.rk.worker};
 
     uint32_t k = 0;
     bool ok = true;
 #pragma unroll 1
-    for (; ok && tile < c.full_tiles; tile += stride, ++k)
-        ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, &tmap, a, c, k, tile, tile + ahead,
-                                                                 box_bytes, local_bucket, scale_writer);
-#pragma unroll 1
-    for (; ok && tile < a.ntiles; tile += stride, ++k)
-        ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, &tmap, a, c, k, tile, tile + ahead,
-                                                                  box_bytes, local_bucket, scale_writer);
+    for (; ok && tile < a.ntiles; tile += stride, ++k) {
+        auto refill = [&](uint32_t stage, uint32_t bar) {
+            const uint32_t next_tile = tile + ahead;
+            if (next_tile < a.ntiles) {
+                mbar_expect_tx(bar, box_bytes);
+                tma_load_2d(stage, &tmap, 0, (int)(next_tile * a.tile_rows), bar);
+            }
+        };
+        if (tile < c.full_tiles)
+            ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+                                                                     local_bucket, scale_writer);
+        else
+            ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+                                                                      local_bucket, scale_writer);
+    }
     if (!ok) {
         // A copy never landed: record it, then give the copies still in flight (the one that was
         // being waited for and those issued after it) a last bounded chance to finish before the
@@ -313,6 +331,84 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
             atomicAdd(timeouts, 1u);
             uint32_t j = k - 1, tl = tile - stride;
             for (int s = 0; s < kQuantStages && tl < a.ntiles; ++s, ++j, tl += stride)
+                mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1);
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Several workers' gradients in ONE launch (the server-side simulation of P workers, or a host
+// with several model replicas on one device).  The launch's fixed costs - scheduling the grid,
+// the first tiles' DRAM latency, the last tiles' drain - are paid once instead of once per
+// worker.  The tiles of all workers form one sequence v = worker * ntiles + tile, walked exactly
+// like the one-worker kernel walks its tiles; every tile is encoded by the same code, so worker
+// w's outputs are bit-identical to a one-worker launch with worker id first_worker + w.
+// ---------------------------------------------------------------------------------------
+struct WorkerTable {
+    CUtensorMap map[kMaxWorkers];
+    const void* grad[kMaxWorkers];
+    uint32_t* codes[kMaxWorkers];
+    float* scales[kMaxWorkers];
+};
+
+template <int BITS, int DTYPE, bool SHUFFLE>
+__global__ void __launch_bounds__(128, 4)
+quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_constant__ QuantizeArgs a,
+                        const __grid_constant__ TmaQuantizeConsts c, uint32_t total_tiles,
+                        unsigned int* __restrict__ timeouts)
+{
+    constexpr int THREADS = 128;
+    using Shared = TmaQuantizeShared<DTYPE, THREADS>;
+    constexpr int kQuantStages = Shared::kStages;
+    __shared__ Shared sh;
+
+    const uint32_t t = threadIdx.x;
+    const uint32_t stride = gridDim.x;
+    const uint32_t box_bytes = a.tile_rows * Shared::kRowBytes;
+    if (t == 0) {
+        for (int s = 0; s < kQuantStages; ++s) mbar_init(smem_u32(&sh.bar[s]), 1);
+        fence_barrier_init();
+    }
+    if (t < 3 * (THREADS / 32)) (&sh.slots[0][0])[t] = 0u;
+    grid_dependency_release();
+    __syncthreads();
+    grid_dependency_wait();            // nothing above touches global memory
+
+    auto load_tile = [&](uint32_t v, uint32_t stage, uint32_t bar) {     // thread 0 only
+        if (v < total_tiles) {
+            const uint32_t w = v / a.ntiles;
+            mbar_expect_tx(bar, box_bytes);
+            tma_load_2d(stage, &tab.map[w], 0, (int)((v - w * a.ntiles) * a.tile_rows), bar);
+        }
+    };
+    uint32_t v = blockIdx.x;
+    if (t == 0)
+        for (uint32_t s = 0; s < (uint32_t)kQuantStages; ++s)
+            load_tile(v + s * stride, smem_u32(sh.stage[s]), smem_u32(&sh.bar[s]));
+    const uint32_t local_bucket = t / a.rows_per_bucket;
+    const bool scale_writer = (t % a.rows_per_bucket) == 0;
+    const uint32_t ahead = kQuantStages * stride;
+
+    uint32_t k = 0;
+    bool ok = true;
+#pragma unroll 1
+    for (; ok && v < total_tiles; v += stride, ++k) {
+        const uint32_t w = v / a.ntiles, tile = v - w * a.ntiles;
+        const WorkerView wv = {&tab.map[w], tab.grad[w], tab.codes[w], tab.scales[w], c.rk.worker + w};
+        auto refill = [&](uint32_t stage, uint32_t bar) { load_tile(v + ahead, stage, bar); };
+        if (tile < c.full_tiles)
+            ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+                                                                     local_bucket, scale_writer);
+        else
+            ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+                                                                      local_bucket, scale_writer);
+    }
+    if (!ok) {                         // as in the one-worker kernel
+        if (t == 0) {
+            atomicAdd(timeouts, 1u);
+            uint32_t j = k - 1, vl = v - stride;
+            for (int s = 0; s < kQuantStages && vl < total_tiles; ++s, ++j, vl += stride)
                 mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1);
         }
         __syncthreads();
@@ -382,12 +478,11 @@ static bool tma_path_applies(uint64_t n, uint64_t rpb, uint64_t elem_offset)
     return ((rpb & (rpb - 1)) == 0 && rpb <= 32) || rpb % 32 == 0;
 }
 
-cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64_t bucket,
-                                  uint64_t seed, uint32_t* codes, float* scales, int dtype,
-                                  uint32_t worker, uint32_t step, uint64_t elem_offset,
-                                  cudaStream_t stream)
+// Fills the arguments every fused kernel shares.  Returns rows per bucket.
+static uint64_t fill_args(QuantizeArgs& a, const void* grad, uint64_t n, int bits, uint64_t bucket,
+                          uint64_t seed, uint32_t* codes, float* scales, uint32_t worker, uint32_t step,
+                          uint64_t elem_offset)
 {
-    QuantizeArgs a;
     a.grad = grad; a.codes = codes; a.scales = scales;
     a.n = n;
     a.nrows = (n + 31) / 32;
@@ -402,27 +497,46 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
     a.key.seed_lo = (uint32_t)seed; a.key.seed_hi = (uint32_t)(seed >> 32);
     a.key.worker = worker; a.key.step = step;
     a.nrows_full = n / 32;
+    return rpb;
+}
+
+// Tile shape and constants of the TMA kernels (tma_path_applies() holds).  Returns the CTA size,
+// or 0 if the tile count does not fit.
+static int fill_tma_args(QuantizeArgs& a, TmaQuantizeConsts& c, uint64_t rpb)
+{
+    const int threads = rpb <= 128 ? 128 : 256;
+    a.buckets_per_tile = (uint32_t)(threads / rpb);
+    a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
+    const uint64_t nt = (a.nrows + a.tile_rows - 1) / a.tile_rows;
+    if (nt > 0x7FFFFFFFull) return 0;
+    a.ntiles = (uint32_t)nt;
+    uint32_t k0 = a.key.seed_lo, k1 = a.key.seed_hi;
+    for (int r = 0; r < 10; ++r) {
+        c.rk.k0[r] = k0; c.rk.k1[r] = k1;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    c.rk.worker = a.key.worker; c.rk.step = a.key.step;
+    c.full_tiles = a.tile_rows == (uint32_t)threads ? (uint32_t)(a.nrows_full / a.tile_rows) : 0u;
+    c.blk0_lo = (uint32_t)(a.elem_offset >> 3); c.blk0_hi = (uint32_t)(a.elem_offset >> 35);
+    return threads;
+}
+
+cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64_t bucket,
+                                  uint64_t seed, uint32_t* codes, float* scales, int dtype,
+                                  uint32_t worker, uint32_t step, uint64_t elem_offset,
+                                  cudaStream_t stream)
+{
+    QuantizeArgs a;
+    const uint64_t rpb = fill_args(a, grad, n, bits, bucket, seed, codes, scales, worker, step, elem_offset);
     if (tma_path_applies(n, rpb, elem_offset)) {
-        const int threads = rpb <= 128 ? 128 : 256;
-        a.buckets_per_tile = (uint32_t)(threads / rpb);
-        a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
-        const uint64_t nt = (a.nrows + a.tile_rows - 1) / a.tile_rows;
-        if (nt > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-        a.ntiles = (uint32_t)nt;
+        TmaQuantizeConsts c;
+        const int threads = fill_tma_args(a, c, rpb);
+        if (threads == 0) return cudaErrorInvalidValue;
         CUtensorMap map;
         const char* why = nullptr;
         unsigned int* timeouts = wait_timeout_counter();
         if (timeouts != nullptr &&
             encode_rows_map(&map, grad, a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why)) {
-            TmaQuantizeConsts c;
-            uint32_t k0 = a.key.seed_lo, k1 = a.key.seed_hi;
-            for (int r = 0; r < 10; ++r) {
-                c.rk.k0[r] = k0; c.rk.k1[r] = k1;
-                k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
-            }
-            c.rk.worker = worker; c.rk.step = step;
-            c.full_tiles = a.tile_rows == (uint32_t)threads ? (uint32_t)(a.nrows_full / a.tile_rows) : 0u;
-            c.blk0_lo = (uint32_t)(elem_offset >> 3); c.blk0_hi = (uint32_t)(elem_offset >> 35);
             const bool shuffle = rpb <= 32;
             switch (bits) {
                 case 1: return launch_tma_bits<1>(map, a, c, dtype, threads, shuffle, timeouts, stream);
@@ -453,6 +567,89 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
         case 6: return launch_bits<6>(a, dtype, aligned, (unsigned)ntiles, stream);
         case 7: return launch_bits<7>(a, dtype, aligned, (unsigned)ntiles, stream);
         case 8: return launch_bits<8>(a, dtype, aligned, (unsigned)ntiles, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+template <int BITS, int DTYPE, bool SHUFFLE>
+static cudaError_t launch_workers_inst(const WorkerTable& tab, const QuantizeArgs& a,
+                                       const TmaQuantizeConsts& c, uint32_t total_tiles,
+                                       unsigned int* timeouts, cudaStream_t stream)
+{
+    auto kernel = quantize_workers_kernel<BITS, DTYPE, SHUFFLE>;
+    static int grid_cap[64] = {};                  // per device; 0 = not yet queried
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (grid_cap[dev] == 0) {
+        int occ = 0, sms = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, 128, 0);
+        if (err != cudaSuccess) return err;
+        err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (err != cudaSuccess) return err;
+        grid_cap[dev] = sms * (occ > 0 ? occ : 1);
+    }
+    unsigned grid = (unsigned)grid_cap[dev];
+    if (grid > total_tiles) grid = total_tiles;
+    return launch_pdl(kernel, grid, 128, stream, tab, a, c, total_tiles, timeouts);
+}
+
+template <int BITS>
+static cudaError_t launch_workers_bits(const WorkerTable& tab, const QuantizeArgs& a,
+                                       const TmaQuantizeConsts& c, uint32_t total_tiles, int dtype,
+                                       bool shuffle, unsigned int* timeouts, cudaStream_t stream)
+{
+    if (dtype == 0)
+        return shuffle ? launch_workers_inst<BITS, 0, true>(tab, a, c, total_tiles, timeouts, stream)
+                       : launch_workers_inst<BITS, 0, false>(tab, a, c, total_tiles, timeouts, stream);
+    return shuffle ? launch_workers_inst<BITS, 1, true>(tab, a, c, total_tiles, timeouts, stream)
+                   : launch_workers_inst<BITS, 1, false>(tab, a, c, total_tiles, timeouts, stream);
+}
+
+bool quantize_workers_applies(int W, uint64_t n, uint64_t bucket, uint64_t elem_offset)
+{
+    if (W < 2 || W > kMaxWorkers || n == 0) return false;
+    const uint64_t nrows = (n + 31) / 32;
+    const uint64_t rpb = (bucket >= n) ? nrows : bucket / 32;
+    if ((bucket < n ? bucket : n) > (uint64_t)kMaxFusedBucket) return false;
+    if (!tma_path_applies(n, rpb, elem_offset) || rpb > 128) return false;
+    const uint64_t tile_rows = (128 / rpb) * rpb;
+    const uint64_t nt = (nrows + tile_rows - 1) / tile_rows;
+    return nt * (uint64_t)W <= 0x7FFFFFFFull;
+}
+
+cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n, int bits,
+                                    uint64_t bucket, uint64_t seed, uint32_t* const* codes,
+                                    float* const* scales, int dtype, uint32_t first_worker,
+                                    uint32_t step, uint64_t elem_offset, cudaStream_t stream)
+{
+    QuantizeArgs a;
+    const uint64_t rpb = fill_args(a, grads[0], n, bits, bucket, seed, codes[0], scales[0], first_worker,
+                                   step, elem_offset);
+    TmaQuantizeConsts c;
+    if (fill_tma_args(a, c, rpb) != 128) return cudaErrorInvalidValue;
+    unsigned int* timeouts = wait_timeout_counter();
+    if (timeouts == nullptr) return cudaErrorNotSupported;
+    WorkerTable tab;
+    memset(&tab, 0, sizeof(tab));
+    for (int w = 0; w < W; ++w) {
+        const char* why = nullptr;
+        if (!encode_rows_map(&tab.map[w], grads[w], a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why))
+            return cudaErrorNotSupported;
+        tab.grad[w] = grads[w]; tab.codes[w] = codes[w]; tab.scales[w] = scales[w];
+    }
+    const uint32_t total_tiles = a.ntiles * (uint32_t)W;
+    const bool shuffle = rpb <= 32;
+    switch (bits) {
+        case 1: return launch_workers_bits<1>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 2: return launch_workers_bits<2>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 3: return launch_workers_bits<3>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 4: return launch_workers_bits<4>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 5: return launch_workers_bits<5>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 6: return launch_workers_bits<6>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 7: return launch_workers_bits<7>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+        case 8: return launch_workers_bits<8>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
     }
     return cudaErrorInvalidValue;
 }
