@@ -5,17 +5,20 @@
 
 Workload (the configuration the headline metric is quoted on): one flat gradient of
 n = 25,000,000 fp32 per worker, W = 8 simulated workers, iid Laplace(0, 1e-4), bucket 2048,
-bit widths 1..8.  One step = one pass of the whole path for every bit width: 8 x W quantize
-launches (each reads a distinct 100 MB gradient) followed by 8 fused server launches (each
-reads W code buffers and updates its own 100 MB parameter replica), so every launch reads
-inputs that have been evicted from L2 (> 1.7 GB cycles between reuses).
+bit widths 1..8.  One step = one pass of the whole path for every bit width: the quantize phase
+(per bit width one mqg_quantize_workers launch over all W gradients, 800 MB; or, with
+--quantize-launch per-worker, W mqg_quantize launches of 100 MB each) followed by 8 fused server
+launches (each reads W code buffers and updates its own 100 MB parameter replica), so every
+launch reads inputs that have been evicted from L2 (> 1.7 GB cycles between reuses).
 
 Prints ONE JSON line (rank 0).  `value` is GB/s of fp32 gradient through the whole path
 (8 * W * 4n bytes per step / step time) with all inputs resident in HBM; `e2e` is the same
 metric with the gradients starting in pinned host memory and the updated parameters read
-back, copies inside the timed region; `roofline` describes the dominant kernel
-(quantize_pack_kernel); `per_bits` lists both kernels for every bit width; `cpu_baseline` is
-the scalar CPU checker timed on a bounded sample of the same workload.
+back, copies inside the timed region; `roofline` describes the dominant kernel (the quantize
+kernel) and `roofline_server` the fused server kernel, both from events at the phase boundaries
+inside the timed region; `per_bits` lists both kernels for every bit width from a second,
+instrumented pass with events around every launch group; `cpu_baseline` is the scalar CPU
+checker timed on a bounded sample of the same workload.
 
 --impl reference times the CPU checker alone (rank 0 only).
 With --gpus N > 1 (under torchrun) every rank runs an independent replica of the workload
@@ -310,7 +313,14 @@ def run_ours(args):
         check(lib.mqg_server_step(code_tab[b], scale_tab[b], W, b, n, B, params[b].data_ptr(), LR,
                                   None, sptr))
 
-    def step(step_no, events=None):
+    def step(step_no, phases=None, events=None):
+        """One pass of the whole path.  `phases`: three events per step (start, quantize phase done,
+        server phase done).  `events`: one pair per launch group instead (the instrumented pass
+        after the timed region; an event between two launches keeps the second from starting
+        while the first drains, so those times are a little longer than in the timed region)."""
+        if phases is not None:
+            p0 = torch.cuda.Event(enable_timing=True)
+            p0.record(stream)
         for b in ALL_BITS:
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -319,6 +329,9 @@ def run_ours(args):
             if events is not None:
                 e1.record(stream)
                 events.append(("q", b, e0, e1))
+        if phases is not None:
+            p1 = torch.cuda.Event(enable_timing=True)
+            p1.record(stream)
         for b in ALL_BITS:
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -327,6 +340,10 @@ def run_ours(args):
             if events is not None:
                 e1.record(stream)
                 events.append(("s", b, e0, e1))
+        if phases is not None:
+            p2 = torch.cuda.Event(enable_timing=True)
+            p2.record(stream)
+            phases.append((p0, p1, p2))
 
     def e2e_step(step_no):
         for b in ALL_BITS:
@@ -349,19 +366,27 @@ def run_ours(args):
     # ---- device-resident timing
     for i in range(args.warmup):
         step(i)
-    events = []
+    phases = []
     barrier()
     with ClockSampler(local_rank) as clocks:
         t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_begin.record(stream)
         for i in range(args.steps):
-            step(args.warmup + i, events)
+            step(args.warmup + i, phases=phases)
         t_end.record(stream)
         barrier()
     total_ms = max_over_ranks(t_begin.elapsed_time(t_end))
     ms_per_step = total_ms / args.steps
     grad_bytes_per_step = len(ALL_BITS) * W * 4 * n
     value = whole_job_gbs(world, grad_bytes_per_step, ms_per_step)
+    q_phase_s = float(np.mean([p0.elapsed_time(p1) for p0, p1, _ in phases])) * 1e-3
+    s_phase_s = float(np.mean([p1.elapsed_time(p2) for _, p1, p2 in phases])) * 1e-3
+
+    # ---- per bit width: the same steps again with events around every launch group
+    events = []
+    for i in range(args.steps):
+        step(args.warmup + args.steps + i, events=events)
+    torch.cuda.synchronize()
 
     # the other way of launching the quantize phase, timed on its own for comparison
     other = quantize_per_worker if batched else quantize_batched
@@ -404,14 +429,17 @@ def run_ours(args):
             "wire_bytes_per_worker": mqg.mqg_wire_bytes(n, b, B),
             ("quantize_us_per_worker_launches" if batched else "quantize_us_one_launch"): other_ms[b] / W * 1e3,
         })
-    q_achieved = q_bytes_total / q_time_total / 1e9
-    s_achieved = s_bytes_total / s_time_total / 1e9
+    # the roofline figures come from the timed region: bytes of a phase / its duration
+    q_achieved = q_bytes_total / q_phase_s / 1e9
+    s_achieved = s_bytes_total / s_phase_s / 1e9
+    q_time_total, s_time_total = q_phase_s, s_phase_s
     q_kernel = "quantize_workers_kernel" if batched else "quantize_tma_kernel"
     q_per_launch = W if batched else 1     # gradients one launch encodes
     roofline = {"kernel": "%s (all bit widths, %d launches per step, %d gradient(s) of n per launch)"
                           % (q_kernel, len(ALL_BITS) * q_launches, q_per_launch),
                 "bound": "hbm", "achieved": q_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
                 "unit": "GB/s", "frac": q_achieved / peak,
+                "avg_launch_us": q_phase_s / (len(ALL_BITS) * q_launches) * 1e6,
                 "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n * q_per_launch,
                 "traffic_note": "dram read+write bytes per element of a K=4 launch from the ncu capture in "
                                 "profiles/quantize_tma_kernel_b4_n32M.md (n=33.5M; the batched kernel runs the "
@@ -420,7 +448,8 @@ def run_ours(args):
                 "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
     roofline_server = {"kernel": "server_tma_kernel (fused step, all bit widths, %d launches per step)" % len(ALL_BITS),
                        "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
-                       "unit": "GB/s", "frac": s_achieved / peak, "traffic": None}
+                       "unit": "GB/s", "frac": s_achieved / peak,
+                       "avg_launch_us": s_phase_s / len(ALL_BITS) * 1e6, "traffic": None}
 
     # ---- end to end from pinned host buffers
     e2e_steps = max(1, min(args.steps, 3))
