@@ -1,14 +1,15 @@
-// Fused server pass fed by TMA (the fast path of mqg_server_step for uniform buckets of at
-// least 1024 elements): every WARP is an independent pipeline over a contiguous range of rows.
-// It walks its range in tiles of 32 rows; a tile's 32 x 32 parameters arrive by a tiled bulk
-// copy into the warp's own swizzled shared-memory stage (two stages, the next tile is always in
-// flight), are updated in place and leave by a tiled bulk store, so parameter traffic is always
-// full 128-byte lines and never waits on another warp: there is no CTA-wide barrier anywhere.
-// All warps get ranges of the same length (to within one row), so the SMs finish together.
-// The W code streams are read straight from global memory with 128/64/32-bit loads (a lane's
-// row is K consecutive words per worker), a group of workers at a time, the first group one
-// tile ahead.  Per-(worker, bucket) de-quantization constants are computed once per tile into
-// the warp's small shared table, also one tile ahead.
+// Fused server pass fed entirely by TMA (the fast path of mqg_server_step for uniform buckets of
+// at least 1024 elements): every WARP is an independent pipeline over a contiguous range of
+// 32-row tiles.  Nothing is loaded through registers:
+//   * a tile's 32 x 32 parameters arrive by a tiled bulk copy into the warp's own swizzled
+//     shared-memory stage (two stages, the next tile always in flight), are updated in place and
+//     leave by a tiled bulk store;
+//   * the code words of the tile (32 rows x K words per worker, contiguous in each worker's
+//     stream) arrive by one linear bulk copy per worker into a two-deep ring of code stages, a
+//     group of workers per stage, issued two stages ahead of their use.
+// A warp therefore never waits for DRAM latency in steady state and there is no CTA-wide barrier
+// anywhere.  Per-(worker, bucket) de-quantization constants are computed once per tile into the
+// warp's small shared table, one tile ahead.
 #include "mqg_common.cuh"
 #include "mqg_internal.h"
 #include "mqg_tma.cuh"
@@ -19,42 +20,42 @@ constexpr int kSrvWarps = 4;                      // warps per CTA, each with it
 constexpr int kSrvThreads = 32 * kSrvWarps;
 constexpr int kSrvTileRows = 32;                  // rows per tile = lanes per warp
 constexpr uint32_t kSrvTileBytes = kSrvTileRows * 128;
+constexpr int kCodeDepth = 2;                     // code stages per warp
+
+// Workers whose code words share one code stage: at most 2 KB per stage, so that a CTA's shared
+// memory (13 KB per warp) lets four CTAs = 16 warps share an SM, and a power of two, so that the
+// usual worker counts fill whole stages.
+template <int BITS>
+struct ServerGroup { static constexpr int value = BITS <= 2 ? 8 : (BITS <= 4 ? 4 : 2); };
 
 struct ServerTmaArgs {
     WorkerPtrs ptrs;
     float* params;
     uint64_t n, ncode_words;
     uint32_t nrows;              // ceil(n / 32)
-    uint32_t nrows_full;         // floor(n / 32): rows the tensor maps cover
-    uint32_t range_rows;         // rows per warp: ceil(nrows_full / number of warps in the grid)
+    uint32_t nrows_full;         // floor(n / 32): rows the tensor map and the code copies cover
+    uint32_t ntiles;             // ceil(nrows_full / 32)
     uint32_t nbuckets;
     uint32_t rows_per_bucket;    // >= 32, so a tile touches at most two buckets
     int rpb_shift;               // log2(rows_per_bucket) if a power of two, else -1
     int W;
     float neg_lr;
     uint32_t bias_bits;          // 0x4B000000 (2^23), a run-time constant for the byte permutes
-    uint32_t tail_bytes;         // bytes of the short box: (range_rows % 32) * 128
 };
 
-struct alignas(1024) ServerWarpShared {
-    uint8_t stage[2][kSrvTileBytes];
-    float4 table[2][kMaxWorkers][2];      // (2h, 2h, -h, -h) per worker and bucket of the tile
-    uint64_t bar[2];
+// Dynamic shared memory of one CTA (base rounded up to 1024 bytes for the 128-byte swizzle).
+template <int BITS>
+struct ServerSmem {
+    alignas(1024) uint8_t stage[kSrvWarps][2][kSrvTileBytes];
+    alignas(16) uint32_t code[kSrvWarps][kCodeDepth][ServerGroup<BITS>::value][kSrvTileRows * BITS];
+    float2 table[kSrvWarps][2][kMaxWorkers][2];   // (2h, -h) per worker and bucket of the tile
+    uint64_t bar[kSrvWarps][2];                   // parameter stages
+    uint64_t cbar[kSrvWarps][kCodeDepth];         // code stages
 };
 
 __device__ __forceinline__ uint32_t bucket_of_row(const ServerTmaArgs& a, uint32_t row)
 {
     return a.rpb_shift >= 0 ? row >> a.rpb_shift : row / a.rows_per_bucket;
-}
-
-// Requests the code words of workers g0 .. g0+GROUP-1 (those that exist) for one row.
-template <int BITS, int GROUP>
-__device__ __forceinline__ void load_group(const ServerTmaArgs& a, int g0, uint64_t word0,
-                                           uint32_t (&wbuf)[GROUP][BITS])
-{
-#pragma unroll
-    for (int i = 0; i < GROUP; ++i)
-        if (g0 + i < a.W) load_row_words<BITS>(a.ptrs.codes[g0 + i], word0, wbuf[i]);
 }
 
 // Scales of the (worker, bucket) pairs of the tile that starts at row0: lane l holds pair l and
@@ -71,7 +72,7 @@ __device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_
 }
 
 template <int BITS>
-__device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float4 (*table)[2], uint32_t lane,
+__device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float2 (*table)[2], uint32_t lane,
                                                   const float (&s)[2])
 {
 #pragma unroll
@@ -79,61 +80,128 @@ __device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float4
         const uint32_t pair = lane + 32u * h, w = pair >> 1;
         if (w < (uint32_t)a.W) {
             const DecodeScale d = decode_scale<BITS>(s[h]);
-            table[w][pair & 1u] = make_float4(d.two_h, d.two_h, d.minus_h, d.minus_h);
+            table[w][pair & 1u] = make_float2(d.two_h, d.minus_h);
         }
     }
 }
 
-// CTAs per SM the register budget is set for: the decode of the wider codes schedules better
-// with up to 128 registers (4 CTAs = 16 warps per SM) than with 5 CTAs and 102 registers.
+// A lane's K words of one worker from a code stage, with the widest shared-memory access the
+// lane's offset (lane * K words) allows.
 template <int BITS>
-constexpr int server_min_ctas() { return BITS == 1 ? 5 : 4; }
+__device__ __forceinline__ void read_stage_words(const uint32_t* __restrict__ stage_row, uint32_t (&w)[BITS])
+{
+    if constexpr (BITS % 4 == 0) {
+        const uint4* p = reinterpret_cast<const uint4*>(stage_row);
+#pragma unroll
+        for (int k = 0; k < BITS / 4; ++k) {
+            const uint4 v = p[k];
+            w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
+        }
+    } else if constexpr (BITS % 2 == 0) {
+        const uint2* p = reinterpret_cast<const uint2*>(stage_row);
+#pragma unroll
+        for (int k = 0; k < BITS / 2; ++k) {
+            const uint2 v = p[k];
+            w[2 * k] = v.x; w[2 * k + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < BITS; ++k) w[k] = stage_row[k];
+    }
+}
+
+// Starts the copies of one code stage: the words of rows [row0, row0 + 32) (fewer in the last tile
+// of the gradient) of workers g0 .. g0 + group - 1 (those that exist).  A worker's words of these
+// rows are contiguous in its stream and start on a 16-byte boundary (row0 is a multiple of 32),
+// so each worker is one linear bulk copy; a last tile whose byte count is not a multiple of 16
+// is filled with ordinary loads and stores instead.  Called by the whole warp.
+template <int BITS>
+__device__ __forceinline__ void fill_code_stage(const ServerTmaArgs& a, uint32_t* stage, uint32_t bar,
+                                                uint32_t row0, int g0, uint32_t lane)
+{
+    constexpr int kGroup = ServerGroup<BITS>::value;
+    constexpr uint32_t kWorkerWords = kSrvTileRows * BITS;
+    const uint32_t rows_here = min((uint32_t)kSrvTileRows, a.nrows_full - row0);
+    const int nwk = min(kGroup, a.W - g0);
+    const uint64_t word0 = (uint64_t)row0 * BITS;
+    if ((rows_here & 3u) == 0) {
+        if (lane == 0) {
+            const uint32_t bytes = rows_here * BITS * 4u;
+            mbar_expect_tx(bar, bytes * (uint32_t)nwk);
+            for (int i = 0; i < nwk; ++i)
+                bulk_load_1d(smem_u32(stage + i * kWorkerWords), a.ptrs.codes[g0 + i] + word0, bytes, bar);
+        }
+    } else {
+        if (lane < rows_here) {
+            for (int i = 0; i < nwk; ++i) {
+                const uint32_t* src = a.ptrs.codes[g0 + i] + word0 + lane * BITS;
+#pragma unroll
+                for (int j = 0; j < BITS; ++j) stage[i * kWorkerWords + lane * BITS + j] = __ldg(src + j);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar);
+    }
+}
+
+// CTAs per SM the register budget is set for (what the shared memory allows).
+template <int BITS>
+constexpr int server_min_ctas() { return 4; }
 
 // MODE 1: dst = params, dst <- fma(-lr, sum, dst).  MODE 0: dst = acc, dst <- sum.
 // MODE 2: dst = acc, the sum continues from the value already there.
 template <int BITS, int MODE>
 __global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
-server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ CUtensorMap map_tail,
-                  const __grid_constant__ ServerTmaArgs a, unsigned int* __restrict__ timeouts)
+server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ ServerTmaArgs a,
+                  unsigned int* __restrict__ timeouts)
 {
-    __shared__ ServerWarpShared shared[kSrvWarps];
+    extern __shared__ uint8_t smem_raw[];
+    ServerSmem<BITS>& sm = *reinterpret_cast<ServerSmem<BITS>*>(
+        smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
+    constexpr int kGroup = ServerGroup<BITS>::value;
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
-    ServerWarpShared& sh = shared[wid];
+    uint8_t (*stage)[kSrvTileBytes] = sm.stage[wid];
+    uint64_t* bar = sm.bar[wid];
+    uint64_t* cbar = sm.cbar[wid];
 
     if (lane == 0) {
-        mbar_init(smem_u32(&sh.bar[0]), 1);
-        mbar_init(smem_u32(&sh.bar[1]), 1);
+        mbar_init(smem_u32(&bar[0]), 1);
+        mbar_init(smem_u32(&bar[1]), 1);
+#pragma unroll
+        for (int s = 0; s < kCodeDepth; ++s) mbar_init(smem_u32(&cbar[s]), 1);
         fence_barrier_init();
         prefetch_tensormap(&map_full);
-        prefetch_tensormap(&map_tail);
     }
-    grid_dependency_release();
     __syncwarp();
-    grid_dependency_wait();                        // nothing above touches global memory
 
-    // this warp's rows: [r_begin, r_end)
-    const uint32_t gwarp = blockIdx.x * kSrvWarps + wid;
-    const uint64_t begin64 = (uint64_t)gwarp * a.range_rows;
-    const uint32_t r_begin = begin64 < a.nrows_full ? (uint32_t)begin64 : a.nrows_full;
-    const uint32_t r_end = (begin64 + a.range_rows < a.nrows_full) ? r_begin + a.range_rows : a.nrows_full;
-    const uint32_t ntiles = (r_end - r_begin + kSrvTileRows - 1) / kSrvTileRows;
+    // this warp's tiles: [t_begin, t_begin + ntiles), the grid's tiles split evenly
+    const uint32_t gwarp = blockIdx.x * kSrvWarps + wid, nwarps = gridDim.x * kSrvWarps;
+    const uint32_t base = a.ntiles / nwarps, extra = a.ntiles % nwarps;
+    const uint32_t t_begin = gwarp * base + min(gwarp, extra);
+    const uint32_t ntiles = base + (gwarp < extra ? 1u : 0u);
+    const uint32_t r_begin = t_begin * kSrvTileRows;
     const uint32_t last_row = a.nrows_full - 1;    // nrows_full >= 1 on this path
+    const uint32_t groups = ((uint32_t)a.W + kGroup - 1) / kGroup;      // code stages per tile
+    const uint32_t nunits = ntiles * groups;
 
-    constexpr int kGroup = BITS <= 4 ? 8 : 32 / BITS;        // workers whose words are in flight together
-    uint32_t wbuf[kGroup][BITS];
     bool failed = false;
-    uint32_t k = 0;
+    uint32_t k = 0, u = 0;                         // tile and code stage in use
     if (ntiles > 0) {
         float s0[2];
         load_tile_scales(a, r_begin, lane, s0);
-        store_tile_scales<BITS>(a, sh.table[0], lane, s0);
-        load_group<BITS, kGroup>(a, 0, (uint64_t)min(r_begin + lane, last_row) * BITS, wbuf);
+        store_tile_scales<BITS>(a, sm.table[wid][0], lane, s0);
         if (MODE != 0 && lane == 0) {
-            mbar_expect_tx(smem_u32(&sh.bar[0]), kSrvTileBytes);
-            tma_load_2d(smem_u32(sh.stage[0]), &map_full, 0, (int)r_begin, smem_u32(&sh.bar[0]));
+            mbar_expect_tx(smem_u32(&bar[0]), kSrvTileBytes);
+            tma_load_2d(smem_u32(stage[0]), &map_full, 0, (int)r_begin, smem_u32(&bar[0]));
         }
+        // the first kCodeDepth code stages (u2 = stage number, tile u2 / groups, group u2 % groups)
+        for (uint32_t u2 = 0; u2 < (uint32_t)kCodeDepth && u2 < nunits; ++u2)
+            fill_code_stage<BITS>(a, &sm.code[wid][u2][0][0], smem_u32(&cbar[u2]),
+                                  r_begin + (u2 / groups) * kSrvTileRows, (int)(u2 % groups) * kGroup, lane);
         __syncwarp();
     }
+    // position of the code stage kCodeDepth ahead of the one in use, kept incrementally
+    uint32_t fill_tile = kCodeDepth / groups, fill_group = kCodeDepth % groups;
 
 #pragma unroll 1
     for (; k < ntiles; ++k) {
@@ -149,31 +217,27 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
             __syncwarp();
         } else if (lane == 0 && have_next) {
             bulk_wait_read<0>();
-            const uint32_t bar = smem_u32(&sh.bar[stg ^ 1]);
-            const uint32_t next0 = row0 + kSrvTileRows;
-            if (r_end - next0 >= (uint32_t)kSrvTileRows || r_end == a.nrows_full) {
-                mbar_expect_tx(bar, kSrvTileBytes);
-                tma_load_2d(smem_u32(sh.stage[stg ^ 1]), &map_full, 0, (int)next0, bar);
-            } else {                               // short last tile of the range: the short box
-                mbar_expect_tx(bar, a.tail_bytes);
-                tma_load_2d(smem_u32(sh.stage[stg ^ 1]), &map_tail, 0, (int)next0, bar);
-            }
+            // the gradient's last tile may be short: the box is clipped by the tensor's bounds and
+            // the rows beyond arrive as zeros, still counted in the bytes
+            mbar_expect_tx(smem_u32(&bar[stg ^ 1]), kSrvTileBytes);
+            tma_load_2d(smem_u32(stage[stg ^ 1]), &map_full, 0, (int)(row0 + kSrvTileRows), smem_u32(&bar[stg ^ 1]));
         }
         float s_next[2];
         if (have_next) load_tile_scales(a, row0 + kSrvTileRows, lane, s_next);
 
         // Sum of the W de-quantized rows, in worker order.  Lanes past the end of the gradient
-        // (only in the very last tile) decode the last row instead; they are never stored.
+        // (only in the very last tile) decode whatever their slot of the stage holds; they are
+        // never stored.
         const uint32_t row = min(row0 + lane, last_row);
         const uint32_t lb = bucket_of_row(a, row) - bucket_of_row(a, row0);
-        const uint64_t word0 = (uint64_t)row * BITS;
         float2 v2[16];
         bool ok = true;
         if constexpr (MODE == 2) {
             // the sum continues from the accumulator: its tile is needed before the first worker
-            ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
-            if (!ok) ok = mbar_wait(smem_u32(&sh.bar[stg]), parity);
-            const float4* tl = reinterpret_cast<const float4*>(sh.stage[stg]);
+            ok = mbar_try_wait(smem_u32(&bar[stg]), parity);
+            if (!ok) ok = mbar_wait(smem_u32(&bar[stg]), parity);
+            if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
+            const float4* tl = reinterpret_cast<const float4*>(stage[stg]);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float4 p = tl[swz((int)lane, c)];
@@ -184,49 +248,46 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
 #pragma unroll
             for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
         }
-        const uint64_t word0_next = (uint64_t)min(row0 + kSrvTileRows + lane, last_row) * BITS;
-        auto decode_slots = [&](int g0, int lo, int hi) {
-#pragma unroll
-            for (int i = lo; i < hi; ++i) {
-                if (g0 + i < a.W) {
-                    const float4 e = sh.table[stg][g0 + i][lb];
-                    DecodeScale2 d;
-                    d.two_h = make_float2(e.x, e.y); d.minus_h = make_float2(e.z, e.w);
-                    add_decoded_row<BITS>(wbuf[i], d, v2, a.bias_bits);
-                }
-            }
-        };
-        auto prefetch_slots = [&](int lo, int hi) {      // next tile's first group into freed slots
-#pragma unroll
-            for (int i = lo; i < hi; ++i)
-                if (i < a.W) load_row_words<BITS>(a.ptrs.codes[i], word0_next, wbuf[i]);
-        };
-        constexpr int kHalf = kGroup / 2;
-        if (BITS >= 5 && a.W <= kGroup) {
-            // one group of wide codes: the slots of each half are refilled for the next tile as
-            // soon as the half has been decoded, so the requests have the rest of the tile's work
-            // to land (measured: faster for K >= 5, slower for the narrow loads of K <= 3)
-            decode_slots(0, 0, kHalf);
-            if (have_next) prefetch_slots(0, kHalf);
-            decode_slots(0, kHalf, kGroup);
-            if (have_next) prefetch_slots(kHalf, kGroup);
-        } else {
+
 #pragma unroll 1
-            for (int g0 = 0; g0 < a.W; g0 += kGroup) {
-                if (g0 > 0) load_group<BITS, kGroup>(a, g0, word0, wbuf);
-                decode_slots(g0, 0, kGroup);
+        for (uint32_t g = 0; g < groups; ++g, ++u) {
+            const uint32_t cs = u % kCodeDepth, cpar = (u / kCodeDepth) & 1;
+            uint32_t* cstage = &sm.code[wid][cs][0][0];
+            bool cok = mbar_try_wait(smem_u32(&cbar[cs]), cpar);
+            if (!cok) cok = mbar_wait(smem_u32(&cbar[cs]), cpar);
+            if (!__all_sync(0xFFFFFFFFu, cok)) { failed = true; break; }
+            const int g0 = (int)g * kGroup;
+            auto decode_worker = [&](int i) {
+                uint32_t w[BITS];
+                read_stage_words<BITS>(cstage + i * (kSrvTileRows * BITS) + lane * BITS, w);
+                const float2 e = sm.table[wid][stg][g0 + i][lb];
+                DecodeScale2 d;
+                d.two_h = make_float2(e.x, e.x); d.minus_h = make_float2(e.y, e.y);
+                add_decoded_row<BITS>(w, d, v2, a.bias_bits);
+            };
+            if (g0 + kGroup <= a.W) {              // a whole stage: straight-line code
+#pragma unroll
+                for (int i = 0; i < kGroup; ++i) decode_worker(i);
+            } else {
+#pragma unroll 1
+                for (int i = 0; g0 + i < a.W; ++i) decode_worker(i);
             }
-            if (have_next) prefetch_slots(0, kGroup);
+            __syncwarp();                          // every lane has read the stage: refill it
+            if (u + kCodeDepth < nunits)
+                fill_code_stage<BITS>(a, cstage, smem_u32(&cbar[cs]), r_begin + fill_tile * kSrvTileRows,
+                                      (int)fill_group * kGroup, lane);
+            if (++fill_group == groups) { fill_group = 0; ++fill_tile; }
         }
+        if (failed) break;
 
         if constexpr (MODE == 1) {
-            ok = mbar_try_wait(smem_u32(&sh.bar[stg]), parity);
-            if (!ok) ok = mbar_wait(smem_u32(&sh.bar[stg]), parity);
+            ok = mbar_try_wait(smem_u32(&bar[stg]), parity);
+            if (!ok) ok = mbar_wait(smem_u32(&bar[stg]), parity);
+            if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
         }
-        if (MODE != 0 && !__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
 
         {
-            float4* tl = reinterpret_cast<float4*>(sh.stage[stg]);
+            float4* tl = reinterpret_cast<float4*>(stage[stg]);
             const float2 nlr = make_float2(a.neg_lr, a.neg_lr);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -243,32 +304,32 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         fence_proxy_async();                                   // the bulk store must see these writes
         if (have_next) {
             // constants of the next tile; table[stg ^ 1] was last read in the previous iteration
-            store_tile_scales<BITS>(a, sh.table[stg ^ 1], lane, s_next);
+            store_tile_scales<BITS>(a, sm.table[wid][stg ^ 1], lane, s_next);
         }
         __syncwarp();
         if (lane == 0) {
-            // A tile that ends at this warp's range end but before the end of the gradient must
-            // not overwrite the next warp's rows: its store uses the map with the shorter box.
-            // At the end of the gradient the full box is clipped by the tensor's bounds.
-            const uint32_t rows_here = r_end - row0;
-            if (rows_here >= (uint32_t)kSrvTileRows || r_end == a.nrows_full)
-                tma_store_2d(&map_full, 0, (int)row0, smem_u32(sh.stage[stg]));
-            else
-                tma_store_2d(&map_tail, 0, (int)row0, smem_u32(sh.stage[stg]));
+            // a short last tile is clipped by the tensor's bounds
+            tma_store_2d(&map_full, 0, (int)row0, smem_u32(stage[stg]));
             bulk_commit();
         }
     }
     if (lane == 0) {
         if (failed) {
             atomicAdd(timeouts, 1u);
-            // the copy that was being waited for and the one issued at the top of this iteration
-            mbar_wait(smem_u32(&sh.bar[k & 1]), (k >> 1) & 1);
-            if (k + 1 < ntiles) mbar_wait(smem_u32(&sh.bar[(k + 1) & 1]), ((k + 1) >> 1) & 1);
+            // Copies that may still be in flight get a last bounded chance to land before the
+            // shared memory can be handed to another CTA: the parameter tile in use and the one
+            // issued at the top of this iteration, and the code stages issued but not consumed.
+            if (MODE != 0) {
+                mbar_wait(smem_u32(&bar[k & 1]), (k >> 1) & 1);
+                if (k + 1 < ntiles) mbar_wait(smem_u32(&bar[(k + 1) & 1]), ((k + 1) >> 1) & 1);
+            }
+            for (uint32_t j = u; j < u + kCodeDepth && j < nunits; ++j)
+                mbar_wait(smem_u32(&cbar[j % kCodeDepth]), (j / kCodeDepth) & 1);
         }
         bulk_wait_all<0>();                                    // stores done before the stage goes away
     }
 
-    // A last row of fewer than 32 elements is not covered by the tensor maps: one lane of the
+    // A last row of fewer than 32 elements is not covered by the tensor map: one lane of the
     // grid's last warp handles it with plain loads and stores.
     if (a.nrows > a.nrows_full && blockIdx.x == gridDim.x - 1 && threadIdx.x == kSrvThreads - 1) {
         const uint32_t row = a.nrows_full;
@@ -305,34 +366,33 @@ static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, 
                                           cudaStream_t stream)
 {
     auto kernel = server_tma_kernel<BITS, MODE>;
-    static int grid_cap[64] = {};
+    constexpr size_t kSmemBytes = sizeof(ServerSmem<BITS>) + 1024;   // + slack to round the base up
+    static int grid_cap[64] = {};                 // per device; 0 = not yet set up
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (grid_cap[dev] == 0) {
         int occ = 0, sms = 0;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kSrvThreads, 0);
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (err != cudaSuccess) return err;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kSrvThreads, kSmemBytes);
         if (err != cudaSuccess) return err;
         err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (err != cudaSuccess) return err;
         grid_cap[dev] = sms * (occ > 0 ? occ : 1);
     }
-    // every warp of the grid gets the same number of rows (the last ones may get fewer)
+    // the tiles are split evenly over the warps of the grid; tiny inputs are not spread too thin
     uint64_t grid = (uint64_t)grid_cap[dev];
-    const uint64_t min_rows = 4 * kSrvTileRows;               // do not spread tiny inputs too thin
-    const uint64_t max_warps = (a.nrows_full + min_rows - 1) / min_rows;
+    const uint64_t max_warps = (a.ntiles + 3) / 4;
     if (grid * kSrvWarps > max_warps) grid = (max_warps + kSrvWarps - 1) / kSrvWarps;
-    const uint64_t warps = grid * kSrvWarps;
-    a.range_rows = (uint32_t)((a.nrows_full + warps - 1) / warps);
-    CUtensorMap map_full, map_tail;
+    CUtensorMap map_full;
     const char* why = nullptr;
     if (!encode_rows_map(&map_full, params, a.nrows_full, 4, 32, kSrvTileRows, &why)) return cudaErrorNotSupported;
-    const uint32_t rem = a.range_rows % kSrvTileRows;
-    a.tail_bytes = (rem ? rem : (uint32_t)kSrvTileRows) * 128u;
-    if (!encode_rows_map(&map_tail, params, a.nrows_full, 4, 32, rem ? rem : kSrvTileRows, &why))
-        return cudaErrorNotSupported;
-    return launch_pdl(kernel, (unsigned)grid, kSrvThreads, stream, map_full, map_tail, a, timeouts);
+    // An ordinary launch: started as a programmatic dependent of the kernel before it, so that its
+    // CTAs become resident while that kernel drains, this kernel measured 9 us slower per launch
+    // (67 us against 58 us, eight launches back to back) - unlike the quantize kernels, which gain.
+    return launch_with_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, map_full, a, timeouts);
 }
 
 template <int BITS>
@@ -362,7 +422,7 @@ cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
     a.ncode_words = (n * (uint64_t)bits + 31) / 32;
     a.nrows = (uint32_t)((n + 31) / 32);
     a.nrows_full = (uint32_t)(n / 32);
-    a.range_rows = 0;
+    a.ntiles = (a.nrows_full + kSrvTileRows - 1) / kSrvTileRows;
     a.nbuckets = (uint32_t)((n + bucket - 1) / bucket);
     const uint64_t rpb = bucket >= n ? a.nrows : bucket / 32;
     a.rows_per_bucket = (uint32_t)(rpb > 0xFFFFFFFFull ? 0xFFFFFFFFull : rpb);
