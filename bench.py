@@ -51,9 +51,9 @@ METRIC = "quantize+pack and dequant+accumulate+update GB/s (fp32 grad) per bit w
 UNIT = "GB/s of fp32 gradient through quantize+pack -> unpack+accumulate+update"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per element of quantize_tma_kernel<4> (ncu, n = 33,554,432):
-# (134.25 MB + 7.6 MB) / 33,554,432; writes are partly still in L2 when the kernel ends
-QUANTIZE_DRAM_BYTES_PER_ELEM_K4 = 141.85e6 / 33_554_432
+# dram__bytes_read.sum + dram__bytes_write.sum per element of quantize_workers_kernel<4> (ncu, 4 x 8,388,608
+# elements): (134.25 MB + 7.82 MB) / 33,554,432; writes are partly still in L2 when the kernel ends
+QUANTIZE_DRAM_BYTES_PER_ELEM_K4 = 142.07e6 / 33_554_432
 
 
 def measured_hbm_peak():
@@ -442,9 +442,9 @@ def run_ours(args):
                 "avg_launch_us": q_phase_s / (len(ALL_BITS) * q_launches) * 1e6,
                 "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n * q_per_launch,
                 "traffic_note": "dram read+write bytes per element of a K=4 launch from the ncu capture in "
-                                "profiles/quantize_tma_kernel_b4_n32M.md (n=33.5M; the batched kernel runs the "
-                                "same tile code), scaled to the elements of one launch; algorithmic bytes of "
-                                "that launch: %d" % (quantize_bytes(n, 4, B) * q_per_launch),
+                                "profiles/quantize_workers_kernel_b4_W4_n8M.md (33.5M elements; both quantize "
+                                "kernels run the same tile code), scaled to the elements of one launch; "
+                                "algorithmic bytes of that launch: %d" % (quantize_bytes(n, 4, B) * q_per_launch),
                 "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
     roofline_server = {"kernel": "server_tma_kernel (fused step, all bit widths, %d launches per step)" % len(ALL_BITS),
                        "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
