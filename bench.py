@@ -70,6 +70,11 @@ def quantize_bytes(n, bits, bucket):
     return 4 * n + 4 * ((n * bits + 31) // 32) + 4 * ((n + bucket - 1) // bucket)
 
 
+def requantize_bytes(n, bits, bucket, W):
+    """Algorithmic bytes of one downlink launch: W code streams and scale arrays in, one of each out."""
+    return (W + 1) * quantize_bytes(n, bits, bucket) - (W + 1) * 4 * n
+
+
 def server_bytes(n, bits, bucket, W):
     """Algorithmic bytes of one fused server launch: W code streams + W scale arrays + params r/w."""
     return W * (4 * ((n * bits + 31) // 32) + 4 * ((n + bucket - 1) // bucket)) + 8 * n
@@ -520,6 +525,8 @@ def run_single_kernel(args):
                                                     scales[i % rot], first_worker=0, step=i)
         nbytes = W * quantize_bytes(n, b, B)
     else:
+        if args.kernel == "requantize":
+            rot = 6                                # 8 code buffers of n * bits / 8 bytes per set
         g = torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=0)).cuda()
         codes = [[torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(W)]
                  for _ in range(rot)]
@@ -528,25 +535,33 @@ def run_single_kernel(args):
         for r in range(rot):
             for w in range(W):
                 mqg.mqg_quantize(g, n, b, B, PHILOX_SEED, codes[r][w], scales[r][w], worker=w, step=r)
-        params = [torch.from_numpy(wl.params(n, 0.05, config=2)).cuda() for _ in range(rot)]
-        launch = lambda i: mqg.mqg_server_step(codes[i % rot], scales[i % rot], W, b, n, B,
-                                               params[i % rot], LR)
-        nbytes = server_bytes(n, b, B, W)
+        if args.kernel == "requantize":
+            out_c = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
+            out_s = [torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(rot)]
+            launch = lambda i: mqg.mqg_server_requantize(codes[i % rot], scales[i % rot], W, b, n, B, 1.0 / W,
+                                                         PHILOX_SEED, out_c[i % rot], out_s[i % rot],
+                                                         worker=W, step=i)
+            nbytes = requantize_bytes(n, b, B, W)
+        else:
+            params = [torch.from_numpy(wl.params(n, 0.05, config=2)).cuda() for _ in range(rot)]
+            launch = lambda i: mqg.mqg_server_step(codes[i % rot], scales[i % rot], W, b, n, B,
+                                                   params[i % rot], LR)
+            nbytes = server_bytes(n, b, B, W)
     torch.cuda.synchronize()
-    times = []
-    for i in range(args.launches):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
+    # two warm-up launches, then all launches back to back between one pair of events
+    for i in range(2):
         launch(i)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1) * 1e-3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.launches):
+        launch(2 + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    avg = e0.elapsed_time(e1) * 1e-3 / args.launches
     peak, kind = measured_hbm_peak()
-    best, med = min(times), float(np.median(times))
     print(json.dumps({"kernel": args.kernel, "bits": b, "n": n, "workers": W, "bucket": B,
-                      "launches": args.launches, "median_us": med * 1e6, "best_us": best * 1e6,
-                      "algorithmic_bytes": nbytes, "median_gbs": nbytes / med / 1e9,
-                      "frac_of_%s_peak" % kind: nbytes / med / 1e9 / peak}))
+                      "launches": args.launches, "avg_us": avg * 1e6, "algorithmic_bytes": nbytes,
+                      "avg_gbs": nbytes / avg / 1e9, "frac_of_%s_peak" % kind: nbytes / avg / 1e9 / peak}))
     return 0
 
 
@@ -560,7 +575,7 @@ def main():
     ap.add_argument("--quantize-launch", choices=["batched", "per-worker"], default="batched",
                     help="the step's quantize phase: one mqg_quantize_workers launch per bit width for all "
                          "workers' gradients, or one mqg_quantize launch per worker")
-    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server"], default=None,
+    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize"], default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--n", type=int, default=1 << 25)

@@ -14,74 +14,105 @@ struct RequantArgs {
     float* scales_out;
     uint64_t n, nrows, nbuckets, ncode_words;
     uint32_t rows_per_bucket, tile_rows, buckets_per_tile;
+    uint32_t full_tiles;         // leading tiles whose 256 rows are all complete
     int W;
     float mean_scale;
-    DrawKey key;
+    uint32_t bias_bits;          // 0x4B000000 (2^23), a run-time constant for the byte permutes
+    RoundKeys rk;                // Philox round keys of the re-quantization's draws
 };
 
-template <int BITS>
-__global__ void __launch_bounds__(kMaxTileRows)
-requantize_kernel(const RequantArgs a)
+// De-quantization constants (2h, -h) per (worker, bucket of the tile), computed once per tile when
+// the tile holds at most kTableBuckets buckets; smaller buckets compute them per row.
+constexpr int kTableBuckets = 32;
+
+// One tile.  FULL: every thread owns a complete row (vector loads, no bounds checks).  TABLE: the
+// de-quantization constants come from the shared table.
+template <int BITS, bool FULL, bool TABLE>
+__device__ __forceinline__ void requantize_tile(const RequantArgs& a, uint32_t* s_bucket,
+                                                float2 (*s_table)[kTableBuckets])
 {
-    __shared__ uint32_t s_bucket[kMaxTileRows];
     const uint32_t t = threadIdx.x;
     const uint64_t row0 = (uint64_t)blockIdx.x * a.tile_rows;
     const uint64_t rows_left = a.nrows - row0;
-    const uint32_t rows = (uint32_t)(rows_left < a.tile_rows ? rows_left : a.tile_rows);
-    const bool active = t < rows;
+    const uint32_t rows = FULL ? a.tile_rows : (uint32_t)(rows_left < a.tile_rows ? rows_left : a.tile_rows);
+    const bool active = FULL || t < rows;
     const uint64_t row = row0 + t;
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const uint64_t bucket = (uint64_t)blockIdx.x * a.buckets_per_tile + local_bucket;
 
     if (t < a.buckets_per_tile) s_bucket[t] = 0u;
+    if (TABLE) {
+        for (uint32_t idx = t; idx < (uint32_t)a.W * a.buckets_per_tile; idx += blockDim.x) {
+            const uint32_t w = idx / a.buckets_per_tile, lbk = idx - w * a.buckets_per_tile;
+            const uint64_t gb = (uint64_t)blockIdx.x * a.buckets_per_tile + lbk;
+            const DecodeScale d = decode_scale<BITS>(gb < a.nbuckets ? __ldg(a.ptrs.scales[w] + gb) : 0.0f);
+            s_table[w][lbk] = make_float2(d.two_h, d.minus_h);
+        }
+    }
     __syncthreads();
 
     float x[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) x[j] = 0.0f;
     if (active) {
         const uint64_t word0 = row * BITS;
         float2 v2[16];
 #pragma unroll
         for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
+#pragma unroll 4
         for (int w = 0; w < a.W; ++w) {
             uint32_t cw[BITS];
+            if (FULL) {
+                load_row_words<BITS>(a.ptrs.codes[w], word0, cw);
+            } else {
 #pragma unroll
-            for (int j = 0; j < BITS; ++j)
-                cw[j] = (word0 + j < a.ncode_words) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
-            const DecodeScale2 d = widen(decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
-            add_decoded_row<BITS>(cw, d, v2);
+                for (int j = 0; j < BITS; ++j)
+                    cw[j] = (word0 + j < a.ncode_words) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
+            }
+            DecodeScale2 d;
+            if (TABLE) {
+                const float2 e = s_table[w][local_bucket];
+                d.two_h = make_float2(e.x, e.x); d.minus_h = make_float2(e.y, e.y);
+            } else {
+                d = widen(decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
+            }
+            add_decoded_row<BITS>(cw, d, v2, a.bias_bits);
         }
-        floats_from_pairs(v2, x);
-        const uint64_t left = a.n - row * 32;              // elements of this row that exist
+        const float2 ms = make_float2(a.mean_scale, a.mean_scale);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) x[j] = ((uint64_t)j < left) ? __fmul_rn(x[j], a.mean_scale) : 0.0f;
+        for (int p = 0; p < 16; ++p) v2[p] = __fmul2_rn(v2[p], ms);
+        floats_from_pairs(v2, x);
+        if (!FULL) {
+            const uint64_t left = a.n - row * 32;          // elements of this row that exist
+#pragma unroll
+            for (int j = 0; j < 32; ++j) x[j] = ((uint64_t)j < left) ? x[j] : 0.0f;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) x[j] = 0.0f;
     }
 
-    const uint32_t mbits = [&] {
-        uint32_t m = __float_as_uint(row_abs_max(x));
-        const uint32_t rpb = a.rows_per_bucket;
-        if ((rpb & (rpb - 1)) == 0 && rpb <= 32) {
-            for (uint32_t d = rpb >> 1; d > 0; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
-            return m;
-        }
+    uint32_t m = __float_as_uint(row_abs_max(x));
+    const uint32_t rpb = a.rows_per_bucket;
+    if ((rpb & (rpb - 1)) == 0 && rpb <= 32) {
+        for (uint32_t d = rpb >> 1; d > 0; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+    } else {
         if (active) atomicMax(&s_bucket[local_bucket], m);
         __syncthreads();
-        return active ? s_bucket[local_bucket] : 0u;
-    }();
+        m = active ? s_bucket[local_bucket] : 0u;
+    }
     if (!active) return;
 
-    float s = __uint_as_float(mbits);
+    float s = __uint_as_float(m);
     if (s < flush_limit()) s = 0.0f;
-    if (t % a.rows_per_bucket == 0 && bucket < a.nbuckets) a.scales_out[bucket] = s;
+    if (t % a.rows_per_bucket == 0 && (FULL || bucket < a.nbuckets)) a.scales_out[bucket] = s;
 
     const EncodeScale es = encode_scale<BITS>(s);
     uint32_t h[16];
-    draw_row_aligned(row * 32, make_round_keys(a.key), h);
+    // Philox block of the row's first element: 4 * row (64-bit; the downlink draws from position 0)
+    draw_row_blocks((uint32_t)(row << 2), (uint32_t)(row >> 30), a.rk, h);
     uint32_t w[BITS];
     encode_pack_row<BITS>(x, es, h, w);
     const uint64_t word0 = row * BITS;
-    if (row * 32 + 32 <= a.n) {
+    if (FULL || row * 32 + 32 <= a.n) {
         store_row_words<BITS>(a.codes_out, word0, w);
     } else {
         mask_row_words<BITS>(w, (int)(a.n - row * 32) * BITS);
@@ -89,6 +120,23 @@ requantize_kernel(const RequantArgs a)
         for (int k = 0; k < BITS; ++k)
             if (word0 + k < a.ncode_words) a.codes_out[word0 + k] = w[k];
     }
+}
+
+template <int BITS, bool TABLE>
+__global__ void __launch_bounds__(kMaxTileRows)
+requantize_kernel(const __grid_constant__ RequantArgs a)
+{
+    __shared__ uint32_t s_bucket[kMaxTileRows];
+    __shared__ float2 s_table[TABLE ? kMaxWorkers : 1][kTableBuckets];
+    if (blockIdx.x < a.full_tiles) requantize_tile<BITS, true, TABLE>(a, s_bucket, s_table);
+    else requantize_tile<BITS, false, TABLE>(a, s_bucket, s_table);
+}
+
+template <int BITS>
+static void launch_requantize_bits(const RequantArgs& a, unsigned grid, cudaStream_t stream)
+{
+    if (a.buckets_per_tile <= (uint32_t)kTableBuckets) requantize_kernel<BITS, true><<<grid, kMaxTileRows, 0, stream>>>(a);
+    else requantize_kernel<BITS, false><<<grid, kMaxTileRows, 0, stream>>>(a);
 }
 
 cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
@@ -106,20 +154,26 @@ cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
     a.buckets_per_tile = (uint32_t)(kMaxTileRows / rpb);
     a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
     a.W = W; a.mean_scale = mean_scale;
-    a.key.seed_lo = (uint32_t)seed; a.key.seed_hi = (uint32_t)(seed >> 32);
-    a.key.worker = worker; a.key.step = step;
+    a.bias_bits = 0x4B000000u;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        a.rk.k0[r] = k0; a.rk.k1[r] = k1;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    a.rk.worker = worker; a.rk.step = step;
     const uint64_t ntiles = (a.nrows + a.tile_rows - 1) / a.tile_rows;
     if (ntiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    a.full_tiles = a.tile_rows == (uint32_t)kMaxTileRows ? (uint32_t)((n / 32) / a.tile_rows) : 0u;
     const unsigned grid = (unsigned)ntiles;
     switch (bits) {
-        case 1: requantize_kernel<1><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 2: requantize_kernel<2><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 3: requantize_kernel<3><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 4: requantize_kernel<4><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 5: requantize_kernel<5><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 6: requantize_kernel<6><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 7: requantize_kernel<7><<<grid, kMaxTileRows, 0, stream>>>(a); break;
-        case 8: requantize_kernel<8><<<grid, kMaxTileRows, 0, stream>>>(a); break;
+        case 1: launch_requantize_bits<1>(a, grid, stream); break;
+        case 2: launch_requantize_bits<2>(a, grid, stream); break;
+        case 3: launch_requantize_bits<3>(a, grid, stream); break;
+        case 4: launch_requantize_bits<4>(a, grid, stream); break;
+        case 5: launch_requantize_bits<5>(a, grid, stream); break;
+        case 6: launch_requantize_bits<6>(a, grid, stream); break;
+        case 7: launch_requantize_bits<7>(a, grid, stream); break;
+        case 8: launch_requantize_bits<8>(a, grid, stream); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
