@@ -456,6 +456,37 @@ def run_ours(args):
                        "unit": "GB/s", "frac": s_achieved / peak,
                        "avg_launch_us": s_phase_s / len(ALL_BITS) * 1e6, "traffic": None}
 
+    # ---- the downlink (outside `value`): the server re-quantizes the mean for the broadcast.  ALU-bound:
+    # per element 4 W + 13 lane operations (per worker 1 extract + 3 fp for the decode and sum; mean, max,
+    # 5 of Philox, 5 of the encode, 1 pack) against 148 SMs x 128 lanes x the SM clock.
+    down_codes = torch.zeros(mqg.mqg_code_words(n, max(ALL_BITS)), dtype=torch.int32, device="cuda")
+    down_scales = torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda")
+
+    def downlink(b, step_no):
+        check(lib.mqg_server_requantize(code_tab[b], scale_tab[b], W, b, n, B, C.c_float(1.0 / W), PHILOX_SEED,
+                                        down_codes.data_ptr(), down_scales.data_ptr(), W, step_no, sptr))
+
+    down_steps = max(3, min(args.steps, 20))
+    for b in ALL_BITS:
+        downlink(b, 0)
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record(stream)
+    for i in range(down_steps):
+        for b in ALL_BITS:                 # every K reads its own 8 code buffers: 900 MB between reuses
+            downlink(b, 1 + i)
+    d1.record(stream)
+    torch.cuda.synchronize()
+    down_us = d0.elapsed_time(d1) * 1e3 / (down_steps * len(ALL_BITS))
+    sm_clock_hz = (clocks.summary().get("sm_mhz") or 1965.0) * 1e6
+    alu_peak = 148 * 128 * sm_clock_hz / 1e9
+    alu_achieved = (4 * W + 13) * n / (down_us * 1e-6) / 1e9
+    downlink_line = {"kernel": "requantize_kernel (mqg_server_requantize, all bit widths, not part of `value`)",
+                     "avg_launch_us": down_us, "grad_gbs": 4 * n * W / (down_us * 1e-6) / 1e9,
+                     "roofline": {"bound": "alu", "achieved": alu_achieved, "peak": alu_peak,
+                                  "unit": "G lane-op/s", "frac": alu_achieved / alu_peak, "traffic": None,
+                                  "peak_kind": "148 SMs x 128 lanes x sampled SM clock",
+                                  "ops_per_element": 4 * W + 13}}
+
     # ---- end to end from pinned host buffers
     e2e_steps = max(1, min(args.steps, 3))
     e2e_step(0)
@@ -483,7 +514,8 @@ def run_ours(args):
             "config": dict(workload_config(), quantize_launch=args.quantize_launch),
             "clocks": clocks.summary(), "e2e": e2e,
             "gpu_launches": args.steps * len(ALL_BITS) * (q_launches + 1),
-            "roofline": roofline, "roofline_server": roofline_server, "per_bits": per_bits,
+            "roofline": roofline, "roofline_server": roofline_server, "downlink": downlink_line,
+            "per_bits": per_bits,
         }
         if cpu is not None:
             line["cpu_baseline"] = cpu

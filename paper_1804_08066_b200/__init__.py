@@ -6,7 +6,7 @@ kernels of libmqgrad.so.  There is no CPU fallback: a missing library or a CPU t
 raises.
 
 Function names and argument order follow the C ABI:
-  mqg_quantize, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
+  mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
