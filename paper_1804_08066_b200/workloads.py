@@ -64,6 +64,29 @@ def student_t_bf16(n: int, scale: float = 1e-4, nu: float = 3.0, zero_frac: floa
     return f32_to_bf16_bits(x)
 
 
+# The CNN of the paper's evaluation (Section 4.1): two 5x5 convolutions, two large fully connected
+# layers and the softmax layer.  Only the two large weight matrices are quantized (99 % of the
+# parameters); they come first in the flat layout used here so that they form two adjacent
+# segments, and everything else follows uncompressed.
+PAPER_CNN_QUANTIZED = [(3136, 2304), (2304, 3840)]
+PAPER_CNN_UNCOMPRESSED = [(5, 5, 3, 64), (64,), (5, 5, 64, 64), (64,), (2304,), (3840,), (3840, 10), (10,)]
+
+
+def paper_cnn_layout():
+    """(seg_off of the two quantized matrices, total elements of the flat gradient)."""
+    sizes = [int(np.prod(s)) for s in PAPER_CNN_QUANTIZED]
+    seg_off = np.zeros(len(sizes) + 1, np.uint64)
+    seg_off[1:] = np.cumsum(sizes)
+    total = int(seg_off[-1]) + sum(int(np.prod(s)) for s in PAPER_CNN_UNCOMPRESSED)
+    return seg_off, total
+
+
+def paper_cnn_gradient(config: int = 6, worker: int = 0) -> np.ndarray:
+    """Flat synthetic gradient of that model: every tensor N(0, sigma_l), sigma_l log-uniform."""
+    sizes = [int(np.prod(s)) for s in PAPER_CNN_QUANTIZED + PAPER_CNN_UNCOMPRESSED]
+    return layered(sizes, config=config, worker=worker)
+
+
 def alexnet_segments():
     """(seg_off, sizes) of the AlexNet-shaped layered gradient, weights and biases in order."""
     sizes = [int(np.prod(s)) for s in ALEXNET_SHAPES]

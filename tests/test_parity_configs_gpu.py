@@ -1,5 +1,6 @@
 """Parity on the remaining workload shapes: the AlexNet-shaped layered gradient with one scale
-per tensor (full size, every element checked) and the 10^9-element bf16 stress shape (checked on
+per tensor and the paper's own CNN with its two large matrices quantized (both full size, every
+element checked), and the 10^9-element bf16 stress shape (checked on
 sampled buckets, which `elem_offset` lets the CPU checker compute in isolation)."""
 from concurrent.futures import ThreadPoolExecutor
 
@@ -42,6 +43,52 @@ def test_alexnet_layers_one_scale_per_tensor(bits):
     p = Guarded(n, torch.float32, fill=p0)
     mqg.mqg_server_step_segments([c.view for c in dcodes], [s.view for s in dscales], W, bits, seg, coff, p.view, 0.05)
     torch.cuda.synchronize()
+    p.check_guards()
+    assert bits_equal(p.numpy(np.float32), p_ref) == 0
+    assert mqg.mqg_device_timeouts() == 0
+
+
+@pytest.mark.parametrize("bits", [2, 5, 8])
+def test_paper_cnn_two_fc_layers_quantized_rest_uncompressed(bits):
+    """The paper's own model (Section 4.1): the two large fully connected matrices (16,072,704
+    elements, one scale each) go through quantize -> server step; the other tensors are applied
+    uncompressed, worker by worker.  Full size, every element checked."""
+    seg, total = wl.paper_cnn_layout()
+    nq = int(seg[-1])
+    assert nq == 16_072_704 and total == 16_224_586
+    coff = np.zeros(3, np.uint64)
+    coff[1:] = np.cumsum([O.code_words(int(seg[j + 1] - seg[j]), bits) for j in range(2)])
+    W, lr = 3, 0.2 / 3
+    xs = [wl.paper_cnn_gradient(worker=w) for w in range(W)]
+    with ThreadPoolExecutor(W) as ex:
+        refs = list(ex.map(lambda w: O.quantize_segments(xs[w][:nq], seg, coff, bits, seed=6, worker=w, step=1),
+                           range(W)))
+    p0 = wl.params(total, 0.05, config=6)
+    p_ref = p0.copy()
+    head = np.ascontiguousarray(p_ref[:nq])
+    O.server_step_segments([r[0] for r in refs], [r[1] for r in refs], bits, seg, coff, head, lr)
+    p_ref[:nq] = head
+    tail = np.ascontiguousarray(p_ref[nq:])
+    for w in range(W):
+        O.apply(tail, xs[w][nq:], lr)
+    p_ref[nq:] = tail
+
+    grads = [to_dev(x) for x in xs]
+    dcodes, dscales = [], []
+    for w in range(W):
+        codes = Guarded(int(coff[-1]), torch.int32)
+        scales = Guarded(2, torch.float32)
+        mqg.mqg_quantize_segments(grads[w], seg, coff, bits, 6, codes.view, scales.view, worker=w, step=1)
+        dcodes.append(codes), dscales.append(scales)
+    p = Guarded(total, torch.float32, fill=p0)
+    mqg.mqg_server_step_segments([c.view for c in dcodes], [s.view for s in dscales], W, bits, seg, coff, p.view, lr)
+    for w in range(W):
+        mqg.mqg_apply(p.view[nq:], grads[w][nq:], lr, total - nq)
+    torch.cuda.synchronize()
+    for w in range(W):
+        dcodes[w].check_guards(), dscales[w].check_guards()
+        assert bits_equal(dscales[w].numpy(np.float32), refs[w][1]) == 0
+        assert np.array_equal(dcodes[w].numpy(np.uint32), refs[w][0])
     p.check_guards()
     assert bits_equal(p.numpy(np.float32), p_ref) == 0
     assert mqg.mqg_device_timeouts() == 0
