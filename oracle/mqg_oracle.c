@@ -20,7 +20,10 @@
  * exactness on dyadic grids; exhaustive enumeration of the 65,536 rounding draws;
  * statistical unbiasedness; exact-rational brute force on <= 16 elements; Philox
  * against an independent library implementation; scale against numpy max.
- * Parity unpinned: the codec as a whole against the paper -- the paper prints no
+ * The (min, max) nearest-rounding variant at the end of the file (readings M1..M4) is
+ * pinned by exact rational arithmetic, dyadic closed forms, the half-step error bound,
+ * monotonicity, end points and saturation.
+ * Parity unpinned: both codecs as a whole against the paper -- the paper prints no
  * worked example, error bound or sample output of Quantize / De-quantize.
  */
 #include <math.h>
@@ -297,5 +300,120 @@ int mqo_server_step_segments(const uint32_t *const *codes, const float *const *s
                              acc_out ? acc_out + seg_off[j] : NULL);
     }
     free(cw); free(sw);
+    return rc;
+}
+
+/* ---- codec variant: (min, max) range with nearest rounding ------------------
+ * The paper prints no codec; the footnote of Section 3.2 refers to a scheme that
+ * maps the range [min, max] of a tensor linearly onto the 2^K codes and rounds to
+ * the nearest one.  The readings this repository fixes for it (M1..M4):
+ *   M1  per bucket lo = min x_i, hi = max x_i (a zero of either sign is stored as +0);
+ *       both are sent: two floats per bucket, ranges[2k] = lo, ranges[2k+1] = hi.
+ *   M2  r = fl(hi - lo); a bucket with r < 2^-96 is constant: every code is 0.
+ *   M3  code = min(L, floor(fma(fl(x - lo), fl(L / r), 1/2))), L = 2^K - 1
+ *       (round half up on the scaled offset; deterministic, no random draws).
+ *   M4  x^ = fma(q, fl(r / L), lo); a constant bucket decodes to lo.
+ * Sum, update and packing are R9, R11, R12 unchanged.
+ */
+void mqo_bucket_ranges(const float *x, uint64_t n, uint64_t bucket, float *ranges)
+{
+    uint64_t nb = (n + bucket - 1) / bucket;
+    for (uint64_t k = 0; k < nb; ++k) {
+        uint64_t b0 = k * bucket, b1 = b0 + bucket;
+        if (b1 > n) b1 = n;
+        float lo = x[b0], hi = x[b0];
+        for (uint64_t i = b0 + 1; i < b1; ++i) {
+            if (x[i] < lo) lo = x[i];
+            if (x[i] > hi) hi = x[i];
+        }
+        ranges[2 * k] = lo + 0.0f;                        /* M1: -0 -> +0 */
+        ranges[2 * k + 1] = hi + 0.0f;
+    }
+}
+
+void mqo_encode_minmax(const float *x, uint64_t n, int bits, uint64_t bucket,
+                       const float *ranges, uint8_t *q)
+{
+    const int L = (1 << bits) - 1;
+    const float Lf = (float)L;
+    const float tiny = ldexpf(1.0f, -96);
+    for (uint64_t i = 0; i < n; ++i) {
+        float lo = ranges[2 * (i / bucket)], hi = ranges[2 * (i / bucket) + 1];
+        float r = hi - lo;                                /* M2, one rounding */
+        if (r < tiny) { q[i] = 0; continue; }
+        float inv = Lf / r;                               /* one rounding */
+        float d = x[i] - lo;                              /* one rounding */
+        float t = fmaf(d, inv, 0.5f);                     /* M3, one rounding */
+        int code = (int)floorf(t);
+        if (code > L) code = L;
+        if (code < 0) code = 0;
+        q[i] = (uint8_t)code;
+    }
+}
+
+void mqo_dequantize_minmax(const uint8_t *q, uint64_t n, int bits, uint64_t bucket,
+                           const float *ranges, float *xhat)
+{
+    const float Lf = (float)((1 << bits) - 1);
+    const float tiny = ldexpf(1.0f, -96);
+    for (uint64_t i = 0; i < n; ++i) {
+        float lo = ranges[2 * (i / bucket)], hi = ranges[2 * (i / bucket) + 1];
+        float r = hi - lo;
+        if (r < tiny) { xhat[i] = lo; continue; }         /* M4, constant bucket */
+        float step = r / Lf;                              /* one rounding */
+        xhat[i] = fmaf((float)q[i], step, lo);            /* one rounding */
+    }
+}
+
+int mqo_quantize_minmax(const void *grad, uint64_t n, int bits, uint64_t bucket,
+                        uint32_t *codes, float *ranges, int dtype)
+{
+    if (bits < 1 || bits > 8 || bucket == 0) return -1;
+    if (n == 0) return 0;
+    float *x = (float *)malloc(n * sizeof(float));
+    uint8_t *q = (uint8_t *)malloc(n);
+    if (!x || !q) { free(x); free(q); return -2; }
+    if (dtype == 1) mqo_widen_bf16((const uint16_t *)grad, n, x);
+    else memcpy(x, grad, n * sizeof(float));
+    mqo_bucket_ranges(x, n, bucket, ranges);
+    mqo_encode_minmax(x, n, bits, bucket, ranges, q);
+    mqo_pack(q, n, bits, codes);
+    free(x); free(q);
+    return 0;
+}
+
+int mqo_dequant_accumulate_minmax(const uint32_t *const *codes, const float *const *ranges, int W,
+                                  int bits, uint64_t n, float *acc, uint64_t bucket, int add_into_acc)
+{
+    if (bits < 1 || bits > 8 || bucket == 0 || W < 1) return -1;
+    if (n == 0) return 0;
+    uint8_t *q = (uint8_t *)malloc(n);
+    float *xhat = (float *)malloc(n * sizeof(float));
+    if (!q || !xhat) { free(q); free(xhat); return -2; }
+    for (int w = 0; w < W; ++w) {
+        mqo_unpack(codes[w], n, bits, q);
+        mqo_dequantize_minmax(q, n, bits, bucket, ranges[w], xhat);
+        if (w == 0 && !add_into_acc) {
+            for (uint64_t i = 0; i < n; ++i) acc[i] = xhat[i];
+        } else {
+            for (uint64_t i = 0; i < n; ++i) acc[i] = acc[i] + xhat[i];
+        }
+    }
+    free(q); free(xhat);
+    return 0;
+}
+
+int mqo_server_step_minmax(const uint32_t *const *codes, const float *const *ranges, int W, int bits,
+                           uint64_t n, uint64_t bucket, float *params, float lr, float *acc_out)
+{
+    if (n == 0) return 0;
+    float *acc = (float *)malloc(n * sizeof(float));
+    if (!acc) return -2;
+    int rc = mqo_dequant_accumulate_minmax(codes, ranges, W, bits, n, acc, bucket, 0);
+    if (rc == 0) {
+        mqo_apply(params, acc, lr, n);
+        if (acc_out) memcpy(acc_out, acc, n * sizeof(float));
+    }
+    free(acc);
     return rc;
 }

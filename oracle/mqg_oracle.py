@@ -217,3 +217,72 @@ def server_step_segments(codes, scales, bits, seg_off, code_off, params, lr, wan
     if rc:
         raise ValueError("mqo_server_step_segments failed: %d" % rc)
     return params, acc
+
+
+# ---- codec variant: (min, max) range with nearest rounding ---------------------------------
+_ranges = _decl("mqo_bucket_ranges", None, _vp, _u64, _u64, _vp)
+_encode_mm = _decl("mqo_encode_minmax", None, _vp, _u64, _int, _u64, _vp, _vp)
+_dequant_mm = _decl("mqo_dequantize_minmax", None, _vp, _u64, _int, _u64, _vp, _vp)
+_quantize_mm = _decl("mqo_quantize_minmax", _int, _vp, _u64, _int, _u64, _vp, _vp, _int)
+_deq_acc_mm = _decl("mqo_dequant_accumulate_minmax", _int, _vp, _vp, _int, _int, _u64, _vp, _u64, _int)
+_server_mm = _decl("mqo_server_step_minmax", _int, _vp, _vp, _int, _int, _u64, _u64, _vp, C.c_float, _vp)
+
+
+def bucket_ranges(x, bucket):
+    """(lo, hi) per bucket, interleaved: ranges[2k] = lo, ranges[2k + 1] = hi."""
+    x = _c(x, np.float32)
+    r = np.empty(2 * num_buckets(x.size, bucket), np.float32)
+    _ranges(_ptr(x), x.size, bucket, _ptr(r))
+    return r
+
+
+def encode_minmax(x, bits, bucket, ranges):
+    x = _c(x, np.float32)
+    ranges = _c(ranges, np.float32)
+    assert ranges.size == 2 * num_buckets(x.size, bucket)
+    q = np.empty(x.size, np.uint8)
+    _encode_mm(_ptr(x), x.size, bits, bucket, _ptr(ranges), _ptr(q))
+    return q
+
+
+def dequantize_minmax(q, bits, bucket, ranges):
+    q = _c(q, np.uint8)
+    ranges = _c(ranges, np.float32)
+    xhat = np.empty(q.size, np.float32)
+    _dequant_mm(_ptr(q), q.size, bits, bucket, _ptr(ranges), _ptr(xhat))
+    return xhat
+
+
+def quantize_minmax(grad, bits, bucket, dtype="f32"):
+    grad = _c(grad, np.uint16 if dtype == "bf16" else np.float32)
+    n = grad.size
+    codes = np.zeros(code_words(n, bits), np.uint32)
+    ranges = np.zeros(2 * num_buckets(n, bucket) if n else 0, np.float32)
+    rc = _quantize_mm(_ptr(grad), n, bits, bucket, _ptr(codes), _ptr(ranges), 1 if dtype == "bf16" else 0)
+    if rc:
+        raise ValueError("mqo_quantize_minmax failed: %d" % rc)
+    return codes, ranges
+
+
+def dequant_accumulate_minmax(codes, ranges, bits, n, bucket, acc=None):
+    W = len(codes)
+    codes, ctab = _ptr_array(codes, np.uint32)
+    ranges, rtab = _ptr_array(ranges, np.float32)
+    add = acc is not None
+    out = np.array(acc, np.float32, copy=True) if add else np.empty(n, np.float32)
+    rc = _deq_acc_mm(ctab, rtab, W, bits, n, _ptr(out), bucket, 1 if add else 0)
+    if rc:
+        raise ValueError("mqo_dequant_accumulate_minmax failed: %d" % rc)
+    return out
+
+
+def server_step_minmax(codes, ranges, bits, n, bucket, params, lr, want_acc=False):
+    assert params.dtype == np.float32 and params.flags.c_contiguous and params.size == n
+    W = len(codes)
+    codes, ctab = _ptr_array(codes, np.uint32)
+    ranges, rtab = _ptr_array(ranges, np.float32)
+    acc = np.empty(n, np.float32) if want_acc else None
+    rc = _server_mm(ctab, rtab, W, bits, n, bucket, _ptr(params), lr, _ptr(acc) if want_acc else None)
+    if rc:
+        raise ValueError("mqo_server_step_minmax failed: %d" % rc)
+    return params, acc

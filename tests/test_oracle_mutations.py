@@ -1,5 +1,5 @@
 """Plants single mistakes in a copy of the CPU checker and verifies that the pin
-suite (tests/test_oracle_pins.py) rejects every one of them.  Everything here runs
+suites (tests/test_oracle_pins.py, tests/test_oracle_minmax_pins.py) reject every one of them.  Everything here runs
 on the CPU; the planted copies are compiled into a temporary directory."""
 import os
 import subprocess
@@ -42,6 +42,27 @@ MUTANTS = [
 ]
 
 
+# mistakes planted in the (min, max) nearest-rounding variant, caught by tests/test_oracle_minmax_pins.py
+MUTANTS_MINMAX = [
+    ("mm_dropped_half", "float t = fmaf(d, inv, 0.5f);", "float t = fmaf(d, inv, 0.0f);"),
+    ("mm_unfused", "float t = fmaf(d, inv, 0.5f);", "float t = d * inv + 0.5f;"),
+    ("mm_levels_2_pow_k", "        float inv = Lf / r;                               /* one rounding */",
+     "        float inv = (Lf + 1.0f) / r;"),
+    ("mm_offset_from_hi", "float d = x[i] - lo;", "float d = hi - x[i];"),
+    ("mm_no_clamp", "if (code > L) code = L;", ""),
+    ("mm_range_uses_abs", "if (x[i] < lo) lo = x[i];", "if (fabsf(x[i]) < lo) lo = x[i];"),
+    ("mm_keeps_minus_zero", "ranges[2 * k] = lo + 0.0f;", "ranges[2 * k] = lo;"),
+    ("mm_hi_lo_swapped", "ranges[2 * k + 1] = hi + 0.0f;\n", "ranges[2 * k + 1] = ranges[2 * k]; ranges[2 * k] = hi + 0.0f;\n"),
+    ("mm_decode_unfused", "xhat[i] = fmaf((float)q[i], step, lo);", "xhat[i] = (float)q[i] * step + lo;"),
+    ("mm_decode_from_hi", "xhat[i] = fmaf((float)q[i], step, lo);", "xhat[i] = fmaf(-(float)q[i], step, hi);"),
+    ("mm_decode_step_per_2_pow_k", "float step = r / Lf;", "float step = r / (Lf + 1.0f);"),
+    ("mm_constant_decodes_to_zero", "if (r < tiny) { xhat[i] = lo; continue; }", "if (r < tiny) { xhat[i] = 0.0f; continue; }"),
+    ("mm_flush_threshold", "        if (r < tiny) { q[i] = 0; continue; }", "        if (r < 1e-20f) { q[i] = 0; continue; }"),
+    ("mm_sum_skips_last_worker", "for (int w = 0; w < W; ++w) {\n        mqo_unpack(codes[w], n, bits, q);\n        mqo_dequantize_minmax",
+     "for (int w = 0; w < W - (W > 2); ++w) {\n        mqo_unpack(codes[w], n, bits, q);\n        mqo_dequantize_minmax"),
+]
+
+
 def _run(args):
     name, old, new, tmpdir = args
     text = open(SRC).read()
@@ -54,14 +75,15 @@ def _run(args):
     subprocess.run(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math", "-fPIC",
                     "-shared", "-o", so, c, "-lm"], check=True)
     env = dict(os.environ, MQG_ORACLE_LIB=so)
+    pins = "test_oracle_minmax_pins.py" if name.startswith("mm_") else "test_oracle_pins.py"
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                        os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+                        os.path.join(ROOT, "tests", pins)],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
     return name, r.returncode, r.stdout[-400:]
 
 
 def test_every_planted_mistake_is_caught(tmp_path):
-    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS]
+    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS + MUTANTS_MINMAX]
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 2)) as ex:
         results = list(ex.map(_run, jobs))
     survivors = [name for name, rc, _ in results if rc == 0]
