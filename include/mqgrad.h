@@ -144,6 +144,33 @@ mqg_status mqg_server_requantize(const uint32_t* const* codes, const float* cons
                                  uint32_t worker, uint32_t step, void* cuda_stream);
 
 /*
+ * Codec variant: the (min, max) range scheme the footnote of Section 3.2 refers to, with nearest
+ * rounding and no random draws.  Per bucket lo = min x, hi = max x (a zero of either sign stored
+ * as +0), r = fl(hi - lo), L = 2^bits - 1:
+ *     code = min(L, floor(fma(fl(x - lo), fl(L / r), 1/2)))      x^ = fma(code, fl(r / L), lo)
+ * a bucket with r < 2^-96 is constant: every code is 0 and every x^ is lo.
+ *   ranges  [out] 2 * mqg_num_buckets(n, bucket) floats, 8-byte aligned: ranges[2b] = lo,
+ *                 ranges[2b + 1] = hi of bucket b
+ *   codes   [out] as mqg_quantize
+ * Buckets of at most 4096 elements take one pass over the gradient; larger ones two.
+ * Errors as mqg_quantize; MQG_ERR_ALIGN for a ranges pointer that is not 8-byte aligned.
+ */
+mqg_status mqg_quantize_minmax(const void* grad, uint64_t n, int bits, uint64_t bucket, uint32_t* codes,
+                               float* ranges, mqg_dtype dtype, void* cuda_stream);
+
+/*
+ * Server side of the variant: mqg_dequant_accumulate and mqg_server_step with x^ as above and the
+ * same ordered sum and fused update.  `ranges` is a HOST array of W device pointers, each laid out
+ * as mqg_quantize_minmax writes it.
+ */
+mqg_status mqg_dequant_accumulate_minmax(const uint32_t* const* codes, const float* const* ranges, int W,
+                                         int bits, uint64_t n, float* acc, uint64_t bucket,
+                                         int add_into_acc, void* cuda_stream);
+mqg_status mqg_server_step_minmax(const uint32_t* const* codes, const float* const* ranges, int W, int bits,
+                                  uint64_t n, uint64_t bucket, float* params, float lr, float* acc_out,
+                                  void* cuda_stream);
+
+/*
  * Per-layer scale ("gradient quantization is applied to these two layers", Section 4.1): the flat
  * gradient is cut into nseg segments; segment j = elements [seg_off[j], seg_off[j+1]) is ONE bucket
  * with scale scales[j], and its bit stream starts on a word boundary at word code_off[j].

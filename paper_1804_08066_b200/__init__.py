@@ -7,7 +7,8 @@ raises.
 
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
-  mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_code_words, mqg_num_buckets,
+  mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_quantize_minmax,
+  mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
 from __future__ import annotations
@@ -52,6 +53,9 @@ def _load() -> C.CDLL:
         "mqg_quantize_workers": (i32, [vp, i32, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
         "mqg_apply": (i32, [vp, vp, f32, u64, vp]),
+        "mqg_quantize_minmax": (i32, [vp, u64, i32, u64, vp, vp, i32, vp]),
+        "mqg_dequant_accumulate_minmax": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
+        "mqg_server_step_minmax": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
         "mqg_server_step": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
         "mqg_server_requantize": (i32, [vp, vp, i32, i32, u64, u64, f32, u64, vp, vp, u32, u32, vp]),
         "mqg_quantize_segments": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
@@ -173,6 +177,28 @@ def mqg_server_step(codes, scales, W: int, bits: int, n: int, bucket: int, param
                                 n, bucket, _dev_ptr(params, "params") if n else None, lr,
                                 _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
                                 _stream()))
+
+
+def mqg_quantize_minmax(grad, n: int, bits: int, bucket: int, codes, ranges) -> None:
+    """(min, max) nearest-rounding variant: writes `codes` and `ranges` (lo, hi per bucket)."""
+    _check(_lib.mqg_quantize_minmax(_dev_ptr(grad, "grad") if n else None, n, bits, bucket,
+                                    _dev_ptr(codes, "codes") if n else None,
+                                    _dev_ptr(ranges, "ranges") if n else None, _grad_dtype(grad), _stream()))
+
+
+def mqg_dequant_accumulate_minmax(codes, ranges, W: int, bits: int, n: int, acc, bucket: int,
+                                  add_into_acc: bool = False) -> None:
+    _check(_lib.mqg_dequant_accumulate_minmax(_ptr_table(codes, "codes"), _ptr_table(ranges, "ranges"),
+                                              W, bits, n, _dev_ptr(acc, "acc") if n else None, bucket,
+                                              1 if add_into_acc else 0, _stream()))
+
+
+def mqg_server_step_minmax(codes, ranges, W: int, bits: int, n: int, bucket: int, params, lr: float,
+                           acc_out=None) -> None:
+    _check(_lib.mqg_server_step_minmax(_ptr_table(codes, "codes"), _ptr_table(ranges, "ranges"), W, bits,
+                                       n, bucket, _dev_ptr(params, "params") if n else None, lr,
+                                       _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
+                                       _stream()))
 
 
 def mqg_server_requantize(codes, scales, W: int, bits: int, n: int, bucket: int, mean_scale: float,

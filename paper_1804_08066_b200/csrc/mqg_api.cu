@@ -28,6 +28,7 @@ mqg_status cuda_fail(const char* what, cudaError_t err)
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
 
 mqg_status check_bits(int bits)
 {
@@ -195,6 +196,72 @@ mqg_status mqg_quantize_workers(const void* const* grads, int W, uint64_t n, int
                                            first_worker + (uint32_t)w, step, elem_offset, cuda_stream);
         if (st != MQG_OK) return st;
     }
+    return MQG_OK;
+}
+
+mqg_status mqg_quantize_minmax(const void* grad, uint64_t n, int bits, uint64_t bucket, uint32_t* codes,
+                               float* ranges, mqg_dtype dtype, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (n == 0) return MQG_OK;
+    if (!grad || !codes || !ranges) return fail(MQG_ERR_INVALID, "grad, codes or ranges is null");
+    if (!aligned16(grad)) return fail(MQG_ERR_ALIGN, "grad not 16-byte aligned");
+    if (!aligned16(codes)) return fail(MQG_ERR_ALIGN, "codes not 16-byte aligned");
+    if (!aligned8(ranges)) return fail(MQG_ERR_ALIGN, "ranges not 8-byte aligned");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const cudaError_t err = mqg::quantize_range_fused_applies(n, bucket)
+        ? mqg::launch_quantize_range_fused(grad, n, bits, bucket, codes, ranges, (int)dtype, stream)
+        : mqg::launch_quantize_range_general(grad, n, bits, bucket, codes, ranges, (int)dtype, stream);
+    if (err != cudaSuccess) return cuda_fail("mqg_quantize_minmax", err);
+    return MQG_OK;
+}
+
+// The variant's worker tables: as check_workers, with the stricter alignment of the range pairs.
+static mqg_status check_range_workers(const uint32_t* const* codes, const float* const* ranges, int W,
+                                      bool empty, mqg::WorkerPtrs* out)
+{
+    if (mqg_status st = check_workers(codes, ranges, W, empty, out)) return st;
+    if (empty) return MQG_OK;
+    for (int w = 0; w < W; ++w)
+        if (!aligned8(ranges[w])) return fail(MQG_ERR_ALIGN, "worker %d: ranges not 8-byte aligned", w);
+    return MQG_OK;
+}
+
+mqg_status mqg_dequant_accumulate_minmax(const uint32_t* const* codes, const float* const* ranges, int W,
+                                         int bits, uint64_t n, float* acc, uint64_t bucket,
+                                         int add_into_acc, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    mqg::WorkerPtrs ptrs;
+    if (mqg_status st = check_range_workers(codes, ranges, W, n == 0, &ptrs)) return st;
+    if (n == 0) return MQG_OK;
+    if (!acc) return fail(MQG_ERR_INVALID, "acc is null");
+    if (!aligned16(acc)) return fail(MQG_ERR_ALIGN, "acc not 16-byte aligned");
+    const cudaError_t err = mqg::launch_server_range(ptrs, W, bits, n, bucket, nullptr, 0.0f, acc,
+                                                     add_into_acc ? 1 : 0,
+                                                     static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_dequant_accumulate_minmax", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_server_step_minmax(const uint32_t* const* codes, const float* const* ranges, int W, int bits,
+                                  uint64_t n, uint64_t bucket, float* params, float lr, float* acc_out,
+                                  void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    mqg::WorkerPtrs ptrs;
+    if (mqg_status st = check_range_workers(codes, ranges, W, n == 0, &ptrs)) return st;
+    if (n == 0) return MQG_OK;
+    if (!params) return fail(MQG_ERR_INVALID, "params is null");
+    if (!aligned16(params)) return fail(MQG_ERR_ALIGN, "params not 16-byte aligned");
+    if (acc_out && !aligned16(acc_out)) return fail(MQG_ERR_ALIGN, "acc_out not 16-byte aligned");
+    const cudaError_t err = mqg::launch_server_range(ptrs, W, bits, n, bucket, params, lr, acc_out, 0,
+                                                     static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_server_step_minmax", err);
     return MQG_OK;
 }
 

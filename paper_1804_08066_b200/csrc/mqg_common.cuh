@@ -201,6 +201,75 @@ __device__ __forceinline__ void encode_pack_row(const float (&x)[32], const Enco
     }
 }
 
+// ---------------------------------------------------------------------------------
+// Codec variant: (min, max) range with nearest rounding.  Per bucket lo = min x, hi = max x
+// (a zero of either sign stored as +0), r = fl(hi - lo); code = min(L, floor(fma(fl(x - lo),
+// fl(L / r), 1/2))); x^ = fma(q, fl(r / L), lo); a bucket with r < 2^-96 is constant: every code
+// is 0 and every x^ is lo.
+// ---------------------------------------------------------------------------------
+
+// Order-preserving map of a float's bit pattern to an unsigned integer (-0 sorts just below +0),
+// so that integer min / max reductions and atomics serve float min / max.
+__device__ __forceinline__ uint32_t ordered_bits(float f)
+{
+    const uint32_t b = __float_as_uint(f);
+    return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t u)
+{
+    return __uint_as_float(u ^ ((u >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+}
+constexpr uint32_t kOrderedMinIdentity = 0xFFFFFFFFu;   // above every float
+constexpr uint32_t kOrderedMaxIdentity = 0x00000000u;   // below every float
+
+__device__ __forceinline__ void row_min_max(const float (&x)[32], float& lo, float& hi)
+{
+    lo = x[0]; hi = x[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j) { lo = fminf(lo, x[j]); hi = fmaxf(hi, x[j]); }
+}
+
+struct RangeEncodeScale {
+    float lo, inv;               // inv = fl(L / r), or 0 for a constant bucket (then t = 1/2, code 0)
+};
+
+template <int BITS>
+__device__ __forceinline__ RangeEncodeScale range_encode_scale(float lo, float hi)
+{
+    constexpr float Lf = (float)((1 << BITS) - 1);
+    RangeEncodeScale e;
+    e.lo = lo;
+    const float r = __fsub_rn(hi, lo);
+    e.inv = r < flush_limit() ? 0.0f : __fdiv_rn(Lf, r);
+    return e;
+}
+
+// Nearest-rounding code of one element as the bit pattern of the float 1.5 * 2^23 + q:
+// t = fma(x - lo, inv, 1/2) >= 1/2 is rounded once, then adding 1.5 * 2^23 with rounding towards
+// minus infinity leaves floor(t) in the low mantissa bits.  For lo <= x <= hi, t < L + 1, so the
+// clamp to L needs no instruction.
+__device__ __forceinline__ uint32_t range_encode_bits(float x, const RangeEncodeScale& e)
+{
+    const float d = __fsub_rn(x, e.lo);
+    const float t = __fmaf_rn(d, e.inv, 0.5f);
+    return __float_as_uint(__fadd_rd(t, 12582912.0f));
+}
+
+template <int BITS>
+__device__ __forceinline__ void range_encode_pack_row(const float (&x)[32], const RangeEncodeScale& e,
+                                                      uint32_t (&w)[BITS])
+{
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const uint32_t c = range_encode_bits(x[j], e);
+        const int o = j * BITS, wi = o >> 5, sh = o & 31;
+        if (sh == 0) w[wi] = c - pack_bias<BITS>(wi);
+        else w[wi] = w[wi] + (c << sh);
+        if (sh + BITS > 32)
+            w[wi + 1] = (c >> (32 - sh)) - pack_bias<BITS>(wi + 1);
+    }
+}
+
 // Code j of a row from its BITS words.
 template <int BITS>
 __device__ __forceinline__ uint32_t unpack_one(const uint32_t (&w)[BITS], int j)
@@ -417,6 +486,18 @@ __device__ __forceinline__ DecodeScale decode_scale(float s)
     return d;
 }
 
+// (min, max) variant: (two_h, minus_h) := (step, lo), step = fl(r / L), 0 for a constant bucket.
+template <int BITS>
+__device__ __forceinline__ DecodeScale range_decode_scale(float lo, float hi)
+{
+    constexpr float Lf = (float)((1 << BITS) - 1);
+    DecodeScale d;
+    const float r = __fsub_rn(hi, lo);
+    d.two_h = r < flush_limit() ? 0.0f : __fdiv_rn(r, Lf);
+    d.minus_h = lo;
+    return d;
+}
+
 // ---------------------------------------------------------------------------------
 // Packed fp32x2 arithmetic of sm_100 (__fadd2_rn, __ffma2_rn on float2): one instruction rounds
 // two independent fp32 lanes, each exactly as the scalar instruction would.  It halves the
@@ -425,10 +506,13 @@ __device__ __forceinline__ DecodeScale decode_scale(float s)
 
 // Two codes at once.  m = the floats 2^23 + q (code merged into the mantissa of 2^23);
 // returns v + x^ for both lanes, each x^ rounded once, then the sum rounded once.
-template <int BITS>
+// RANGE: the (min, max) variant, x^ = fma(q, step, lo): the same two instructions with
+// (two_h, minus_h) := (step, lo) and the offset 2^23 alone.
+template <int BITS, bool RANGE = false>
 __device__ __forceinline__ float2 accumulate2(float2 v, float2 m, float2 two_h, float2 minus_h)
 {
-    constexpr float kNegOff = -(8388608.0f + (float)(((1 << BITS) - 2) / 2));   // -(2^23 + (L - 1) / 2)
+    constexpr float kNegOff = RANGE ? -8388608.0f
+                                    : -(8388608.0f + (float)(((1 << BITS) - 2) / 2));   // -(2^23 + (L - 1) / 2)
     const float2 qi = __fadd2_rn(m, make_float2(kNegOff, kNegOff));             // q - (L - 1) / 2, exact
     return __fadd2_rn(v, __ffma2_rn(qi, two_h, minus_h));
 }
@@ -443,11 +527,11 @@ __device__ __forceinline__ float byte_to_biased(uint32_t v, int byte, uint32_t b
 
 // v2[] <- v2[] + de-quantized row; v2[p] holds the running sums of elements 2p and 2p+1 (+0
 // before the first worker: 0 + x^ is exact, and turns the -0 of a zero-scale bucket into +0).
-template <int BITS>
+template <int BITS, bool RANGE = false>
 __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const DecodeScale2& d,
                                                 float2 (&v2)[16], uint32_t bias = 0x4B000000u)
 {
-    if constexpr (BITS == 1) {
+    if constexpr (BITS == 1 && !RANGE) {
         // x^ = +-s (s = h for one bit): set the sign where the code bit is 0
         const uint32_t sbits = __float_as_uint(-d.minus_h.x);
 #pragma unroll
@@ -461,7 +545,7 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
         if constexpr (BITS == 8) {
 #pragma unroll
             for (int p = 0; p < 16; ++p)
-                v2[p] = accumulate2<8>(v2[p], make_float2(byte_to_biased(w[p >> 1], (2 * p) & 3, bias),
+                v2[p] = accumulate2<8, RANGE>(v2[p], make_float2(byte_to_biased(w[p >> 1], (2 * p) & 3, bias),
                                                           byte_to_biased(w[p >> 1], (2 * p + 1) & 3, bias)), th, mh);
         } else if constexpr (BITS == 4) {
 #pragma unroll
@@ -469,7 +553,7 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
                 const uint32_t lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
 #pragma unroll
                 for (int b = 0; b < 4; ++b)      // elements 8k + 2b (low nibble) and 8k + 2b + 1 (high)
-                    v2[4 * k + b] = accumulate2<4>(v2[4 * k + b],
+                    v2[4 * k + b] = accumulate2<4, RANGE>(v2[4 * k + b],
                                                    make_float2(byte_to_biased(lo, b, bias), byte_to_biased(hi, b, bias)), th, mh);
             }
         } else if constexpr (BITS == 2) {
@@ -480,9 +564,9 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
                 for (int r = 0; r < 4; ++r) t[r] = (w[k] >> (2 * r)) & 0x03030303u;
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {    // element 16k + 4b + r lives in byte b of t[r]
-                    v2[8 * k + 2 * b] = accumulate2<2>(v2[8 * k + 2 * b],
+                    v2[8 * k + 2 * b] = accumulate2<2, RANGE>(v2[8 * k + 2 * b],
                                                        make_float2(byte_to_biased(t[0], b, bias), byte_to_biased(t[1], b, bias)), th, mh);
-                    v2[8 * k + 2 * b + 1] = accumulate2<2>(v2[8 * k + 2 * b + 1],
+                    v2[8 * k + 2 * b + 1] = accumulate2<2, RANGE>(v2[8 * k + 2 * b + 1],
                                                            make_float2(byte_to_biased(t[2], b, bias), byte_to_biased(t[3], b, bias)), th, mh);
                 }
             }
@@ -490,7 +574,7 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
 #pragma unroll
             for (int p = 0; p < 16; ++p) {
                 const uint32_t q0 = unpack_one<BITS>(w, 2 * p), q1 = unpack_one<BITS>(w, 2 * p + 1);
-                v2[p] = accumulate2<BITS>(v2[p], make_float2(__uint_as_float(q0 | bias),
+                v2[p] = accumulate2<BITS, RANGE>(v2[p], make_float2(__uint_as_float(q0 | bias),
                                                              __uint_as_float(q1 | bias)), th, mh);
             }
         }

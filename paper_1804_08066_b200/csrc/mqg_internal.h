@@ -42,6 +42,20 @@ cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n,
                                     float* const* scales, int dtype, uint32_t first_worker,
                                     uint32_t step, uint64_t elem_offset, cudaStream_t stream);
 
+// (min, max) nearest-rounding variant.  ranges[2b] = lo, ranges[2b + 1] = hi of bucket b.
+// Fused one-pass kernel for buckets of at most 4096 elements; otherwise the general launches
+// (ranges by atomics on ordered bits, then encode).
+bool quantize_range_fused_applies(uint64_t n, uint64_t bucket);
+cudaError_t launch_quantize_range_fused(const void* grad, uint64_t n, int bits, uint64_t bucket,
+                                        uint32_t* codes, float* ranges, int dtype, cudaStream_t stream);
+cudaError_t launch_quantize_range_general(const void* grad, uint64_t n, int bits, uint64_t bucket,
+                                          uint32_t* codes, float* ranges, int dtype, cudaStream_t stream);
+// Server pass of the variant: `ptrs.scales[w]` points at worker w's ranges.
+cudaError_t launch_server_range(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                                float* params, float lr, float* acc, int add_into, cudaStream_t stream);
+cudaError_t launch_server_range_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                                    float* dst, float lr, int mode, cudaStream_t stream);
+
 // Two-pass quantize of segments.  scales_base points at the scale of the table's first segment.
 cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, int bits,
                                      uint64_t seed, uint32_t* codes, float* scales_base, int dtype,

@@ -173,6 +173,7 @@ struct TmaQuantizeShared {
     static constexpr int kStages = 2 * THREADS * kRowBytes <= 32768 ? 2 : 1;
     alignas(1024) uint8_t stage[kStages][THREADS * kRowBytes];
     uint32_t slots[3][THREADS / 32];       // bucket maxima, rotating so no reset races a use
+    uint32_t slots_lo[3][THREADS / 32];    // bucket minima of the (min, max) variant, as ordered bits
     alignas(8) uint64_t bar[kStages];
 };
 
@@ -270,7 +271,87 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     return true;
 }
 
-template <int BITS, int DTYPE, int THREADS, bool SHUFFLE>
+// The same tile for the (min, max) nearest-rounding variant: two reductions instead of one, two
+// floats per bucket (ranges[2b] = lo, ranges[2b + 1] = hi), no random draws.  Padding must not
+// take part in the range: the elements a ragged row lacks repeat its first element, and threads
+// without a row contribute the identities.  sh.slots holds maxima, sh.slots_lo minima, both as
+// ordered bits; the kernel initialises them to the identities.
+template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, typename Refill>
+__device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
+                                                    const QuantizeArgs& a, uint32_t k, uint32_t tile,
+                                                    Refill&& refill, uint32_t local_bucket, bool scale_writer)
+{
+    constexpr int kQuantStages = TmaQuantizeShared<DTYPE, THREADS>::kStages;
+    const uint32_t t = threadIdx.x;
+    const uint32_t row = tile * a.tile_rows + t;
+    const bool active = FULL || (t < a.tile_rows && row < (uint32_t)a.nrows);
+    const uint32_t stg = k % kQuantStages, parity = (k / kQuantStages) & 1;
+    const uint32_t bar = smem_u32(&sh.bar[stg]);
+    uint8_t* stage = sh.stage[stg];
+
+    bool ok = mbar_try_wait(bar, parity);
+    if (!ok) ok = mbar_wait(bar, parity);
+
+    float x[32];
+    uint32_t mlo = kOrderedMinIdentity, mhi = kOrderedMaxIdentity;
+    if (active) {
+        if (!FULL && row >= (uint32_t)a.nrows_full)
+            stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
+        read_row_swizzled<DTYPE>(stage, (int)t, x);
+        if (!FULL) {
+            const uint64_t left = a.n - (uint64_t)row * 32;      // >= 1
+#pragma unroll
+            for (int j = 1; j < 32; ++j) x[j] = ((uint64_t)j < left) ? x[j] : x[0];
+        }
+        float lo, hi;
+        row_min_max(x, lo, hi);
+        mlo = ordered_bits(lo); mhi = ordered_bits(hi);
+    }
+    uint32_t* slot_hi = sh.slots[k % 3];
+    uint32_t* slot_lo = sh.slots_lo[k % 3];
+    if (SHUFFLE) {
+        for (uint32_t d = a.rows_per_bucket >> 1; d > 0; d >>= 1) {
+            mlo = min(mlo, __shfl_xor_sync(0xFFFFFFFFu, mlo, d));
+            mhi = max(mhi, __shfl_xor_sync(0xFFFFFFFFu, mhi, d));
+        }
+    } else {
+        mlo = __reduce_min_sync(0xFFFFFFFFu, mlo);
+        mhi = __reduce_max_sync(0xFFFFFFFFu, mhi);
+        if ((t & 31) == 0) { atomicMin(&slot_lo[local_bucket], mlo); atomicMax(&slot_hi[local_bucket], mhi); }
+    }
+    if (__syncthreads_or(!ok)) return false;
+    if (t == 0) refill(smem_u32(stage), bar);                    // every thread has read the stage
+    if (!SHUFFLE) {
+        mlo = slot_lo[local_bucket]; mhi = slot_hi[local_bucket];
+        if (t < THREADS / 32) {                                  // next used by this CTA's tile k + 2
+            sh.slots[(k + 2) % 3][t] = kOrderedMaxIdentity;
+            sh.slots_lo[(k + 2) % 3][t] = kOrderedMinIdentity;
+        }
+    }
+    if (!active) return true;
+
+    // a zero of either sign is stored as +0
+    const float lo = __fadd_rn(from_ordered_bits(mlo), 0.0f), hi = __fadd_rn(from_ordered_bits(mhi), 0.0f);
+    const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
+    if (scale_writer && (FULL || bucket < a.nbuckets))
+        reinterpret_cast<float2*>(wv.scales)[bucket] = make_float2(lo, hi);
+
+    const RangeEncodeScale es = range_encode_scale<BITS>(lo, hi);
+    uint32_t w[BITS];
+    range_encode_pack_row<BITS>(x, es, w);
+    const uint64_t word0 = (uint64_t)row * BITS;
+    if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
+        store_row_words<BITS>(wv.codes, word0, w);
+    } else {
+        mask_row_words<BITS>(w, (int)(a.n - (uint64_t)row * 32) * BITS);
+#pragma unroll
+        for (int j = 0; j < BITS; ++j)
+            if (word0 + j < a.ncode_words) wv.codes[word0 + j] = w[j];
+    }
+    return true;
+}
+
+template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, bool RANGE = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ QuantizeArgs a,
                     const __grid_constant__ TmaQuantizeConsts c, unsigned int* __restrict__ timeouts)
@@ -286,7 +367,10 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
         for (int s = 0; s < kQuantStages; ++s) mbar_init(smem_u32(&sh.bar[s]), 1);
         fence_barrier_init();
     }
-    if (t < 3 * (THREADS / 32)) (&sh.slots[0][0])[t] = 0u;
+    if (t < 3 * (THREADS / 32)) {
+        (&sh.slots[0][0])[t] = 0u;     // = kOrderedMaxIdentity
+        (&sh.slots_lo[0][0])[t] = kOrderedMinIdentity;
+    }
     if (t == 0) prefetch_tensormap(&tmap);
     grid_dependency_release();
     __syncthreads();
@@ -315,12 +399,21 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
                 tma_load_2d(stage, &tmap, 0, (int)(next_tile * a.tile_rows), bar);
             }
         };
-        if (tile < c.full_tiles)
-            ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, tile, refill,
-                                                                     local_bucket, scale_writer);
-        else
-            ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, tile, refill,
-                                                                      local_bucket, scale_writer);
+        if constexpr (RANGE) {
+            if (tile < c.full_tiles)
+                ok = range_quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, k, tile, refill,
+                                                                               local_bucket, scale_writer);
+            else
+                ok = range_quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, k, tile, refill,
+                                                                                local_bucket, scale_writer);
+        } else {
+            if (tile < c.full_tiles)
+                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+                                                                         local_bucket, scale_writer);
+            else
+                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+                                                                          local_bucket, scale_writer);
+        }
     }
     if (!ok) {
         // A copy never landed: record it, then give the copies still in flight (the one that was
@@ -430,12 +523,12 @@ static cudaError_t launch_bits(const QuantizeArgs& a, int dtype, bool aligned, u
     return cudaGetLastError();
 }
 
-template <int BITS, int DTYPE, int THREADS, bool SHUFFLE>
+template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, bool RANGE = false>
 static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a,
                                    const TmaQuantizeConsts& c, unsigned int* timeouts,
                                    cudaStream_t stream)
 {
-    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, SHUFFLE>;
+    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, SHUFFLE, RANGE>;
     static int grid_cap[64] = {};                  // per device; 0 = not yet queried
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -650,6 +743,53 @@ cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n,
         case 6: return launch_workers_bits<6>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
         case 7: return launch_workers_bits<7>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
         case 8: return launch_workers_bits<8>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// ---- (min, max) nearest-rounding variant on the TMA kernel (buckets of at most 128 rows) ----
+template <int BITS>
+static cudaError_t launch_range_bits(const CUtensorMap& map, const QuantizeArgs& a, const TmaQuantizeConsts& c,
+                                     int dtype, bool shuffle, unsigned int* timeouts, cudaStream_t stream)
+{
+    if (dtype == 0)
+        return shuffle ? launch_tma_inst<BITS, 0, 128, true, true>(map, a, c, timeouts, stream)
+                       : launch_tma_inst<BITS, 0, 128, false, true>(map, a, c, timeouts, stream);
+    return shuffle ? launch_tma_inst<BITS, 1, 128, true, true>(map, a, c, timeouts, stream)
+                   : launch_tma_inst<BITS, 1, 128, false, true>(map, a, c, timeouts, stream);
+}
+
+bool quantize_range_fused_applies(uint64_t n, uint64_t bucket)
+{
+    if (n == 0) return false;
+    const uint64_t nrows = (n + 31) / 32;
+    const uint64_t rpb = (bucket >= n) ? nrows : bucket / 32;
+    return tma_path_applies(n, rpb, 0) && rpb <= 128;
+}
+
+cudaError_t launch_quantize_range_fused(const void* grad, uint64_t n, int bits, uint64_t bucket,
+                                        uint32_t* codes, float* ranges, int dtype, cudaStream_t stream)
+{
+    QuantizeArgs a;
+    const uint64_t rpb = fill_args(a, grad, n, bits, bucket, 0, codes, ranges, 0, 0, 0);
+    TmaQuantizeConsts c;
+    if (fill_tma_args(a, c, rpb) != 128) return cudaErrorInvalidValue;
+    unsigned int* timeouts = wait_timeout_counter();
+    if (timeouts == nullptr) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const char* why = nullptr;
+    if (!encode_rows_map(&map, grad, a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why))
+        return cudaErrorNotSupported;
+    const bool shuffle = rpb <= 32;
+    switch (bits) {
+        case 1: return launch_range_bits<1>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 2: return launch_range_bits<2>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 3: return launch_range_bits<3>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 4: return launch_range_bits<4>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 5: return launch_range_bits<5>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 6: return launch_range_bits<6>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 7: return launch_range_bits<7>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 8: return launch_range_bits<8>(map, a, c, dtype, shuffle, timeouts, stream);
     }
     return cudaErrorInvalidValue;
 }

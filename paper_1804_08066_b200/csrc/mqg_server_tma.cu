@@ -59,27 +59,31 @@ __device__ __forceinline__ uint32_t bucket_of_row(const ServerTmaArgs& a, uint32
 }
 
 // Scales of the (worker, bucket) pairs of the tile that starts at row0: lane l holds pair l and
-// pair l + 32 (pair = 2 * worker + bucket-of-tile).
+// pair l + 32 (pair = 2 * worker + bucket-of-tile).  RANGE: the pair's (lo, hi) instead of its
+// scale (the `scales` pointers then address arrays of two floats per bucket).
+template <bool RANGE>
 __device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_t row0, uint32_t lane,
-                                                 float (&s)[2])
+                                                 float2 (&s)[2])
 {
     const uint32_t first = bucket_of_row(a, row0);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const uint32_t pair = lane + 32u * h, w = pair >> 1, b = first + (pair & 1u);
-        s[h] = (w < (uint32_t)a.W && b < a.nbuckets) ? __ldg(a.ptrs.scales[w] + b) : 0.0f;
+        const bool have = w < (uint32_t)a.W && b < a.nbuckets;
+        if (RANGE) s[h] = have ? __ldg(reinterpret_cast<const float2*>(a.ptrs.scales[w]) + b) : make_float2(0.0f, 0.0f);
+        else s[h] = make_float2(have ? __ldg(a.ptrs.scales[w] + b) : 0.0f, 0.0f);
     }
 }
 
-template <int BITS>
+template <int BITS, bool RANGE>
 __device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float2 (*table)[2], uint32_t lane,
-                                                  const float (&s)[2])
+                                                  const float2 (&s)[2])
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const uint32_t pair = lane + 32u * h, w = pair >> 1;
         if (w < (uint32_t)a.W) {
-            const DecodeScale d = decode_scale<BITS>(s[h]);
+            const DecodeScale d = RANGE ? range_decode_scale<BITS>(s[h].x, s[h].y) : decode_scale<BITS>(s[h].x);
             table[w][pair & 1u] = make_float2(d.two_h, d.minus_h);
         }
     }
@@ -150,7 +154,8 @@ constexpr int server_min_ctas() { return 4; }
 
 // MODE 1: dst = params, dst <- fma(-lr, sum, dst).  MODE 0: dst = acc, dst <- sum.
 // MODE 2: dst = acc, the sum continues from the value already there.
-template <int BITS, int MODE>
+// RANGE: the (min, max) nearest-rounding variant (x^ = fma(q, step, lo)).
+template <int BITS, int MODE, bool RANGE>
 __global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
 server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ ServerTmaArgs a,
                   unsigned int* __restrict__ timeouts)
@@ -189,9 +194,9 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     bool failed = false;
     uint32_t k = 0, u = 0;                         // tile and code stage in use
     if (ntiles > 0) {
-        float s0[2];
-        load_tile_scales(a, r_begin, lane, s0);
-        store_tile_scales<BITS>(a, sm.table[wid][0], lane, s0);
+        float2 s0[2];
+        load_tile_scales<RANGE>(a, r_begin, lane, s0);
+        store_tile_scales<BITS, RANGE>(a, sm.table[wid][0], lane, s0);
         if (MODE != 0 && lane == 0) {
             mbar_expect_tx(smem_u32(&bar[0]), kSrvTileBytes);
             tma_load_2d(smem_u32(stage[0]), &map_full, 0, (int)r_begin, smem_u32(&bar[0]));
@@ -224,8 +229,8 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
             mbar_expect_tx(smem_u32(&bar[stg ^ 1]), kSrvTileBytes);
             tma_load_2d(smem_u32(stage[stg ^ 1]), &map_full, 0, (int)(row0 + kSrvTileRows), smem_u32(&bar[stg ^ 1]));
         }
-        float s_next[2];
-        if (have_next) load_tile_scales(a, row0 + kSrvTileRows, lane, s_next);
+        float2 s_next[2];
+        if (have_next) load_tile_scales<RANGE>(a, row0 + kSrvTileRows, lane, s_next);
 
         // Sum of the W de-quantized rows, in worker order.  Lanes past the end of the gradient
         // (only in the very last tile) decode whatever their slot of the stage holds; they are
@@ -265,7 +270,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
                 const float2 e = sm.table[wid][stg][g0 + i][lb];
                 DecodeScale2 d;
                 d.two_h = make_float2(e.x, e.x); d.minus_h = make_float2(e.y, e.y);
-                add_decoded_row<BITS>(w, d, v2, a.bias_bits);
+                add_decoded_row<BITS, RANGE>(w, d, v2, a.bias_bits);
             };
             if (g0 + kGroup <= a.W) {              // a whole stage: straight-line code
 #pragma unroll
@@ -306,7 +311,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         fence_proxy_async();                                   // the bulk store must see these writes
         if (have_next) {
             // constants of the next tile; table[stg ^ 1] was last read in the previous iteration
-            store_tile_scales<BITS>(a, sm.table[wid][stg ^ 1], lane, s_next);
+            store_tile_scales<BITS, RANGE>(a, sm.table[wid][stg ^ 1], lane, s_next);
         }
         __syncwarp();
         if (lane == 0) {
@@ -352,8 +357,10 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
 #pragma unroll
             for (int j = 0; j < BITS; ++j)
                 cw[j] = (word0 + j < a.ncode_words) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
-            const DecodeScale2 d = widen(decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
-            add_decoded_row<BITS>(cw, d, v2);
+            const DecodeScale2 d = widen(RANGE ? range_decode_scale<BITS>(__ldg(a.ptrs.scales[w] + 2 * bucket),
+                                                                          __ldg(a.ptrs.scales[w] + 2 * bucket + 1))
+                                               : decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
+            add_decoded_row<BITS, RANGE>(cw, d, v2);
         }
         float v[32];
         floats_from_pairs(v2, v);
@@ -363,11 +370,11 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     }
 }
 
-template <int BITS, int MODE>
+template <int BITS, int MODE, bool RANGE>
 static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, unsigned int* timeouts,
                                           cudaStream_t stream)
 {
-    auto kernel = server_tma_kernel<BITS, MODE>;
+    auto kernel = server_tma_kernel<BITS, MODE, RANGE>;
     constexpr size_t kSmemBytes = sizeof(ServerSmem<BITS>) + 1024;   // + slack to round the base up
     static int grid_cap[64] = {};                 // per device; 0 = not yet set up
     int dev = 0;
@@ -397,13 +404,13 @@ static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, 
     return launch_with_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, map_full, a, timeouts);
 }
 
-template <int BITS>
+template <int BITS, bool RANGE>
 static cudaError_t launch_server_tma_bits(const void* dst, ServerTmaArgs& a, int mode, unsigned int* timeouts,
                                           cudaStream_t stream)
 {
-    if (mode == 1) return launch_server_tma_inst<BITS, 1>(dst, a, timeouts, stream);
-    if (mode == 2) return launch_server_tma_inst<BITS, 2>(dst, a, timeouts, stream);
-    return launch_server_tma_inst<BITS, 0>(dst, a, timeouts, stream);
+    if (mode == 1) return launch_server_tma_inst<BITS, 1, RANGE>(dst, a, timeouts, stream);
+    if (mode == 2) return launch_server_tma_inst<BITS, 2, RANGE>(dst, a, timeouts, stream);
+    return launch_server_tma_inst<BITS, 0, RANGE>(dst, a, timeouts, stream);
 }
 
 bool server_tma_applies(uint64_t n, uint64_t bucket)
@@ -414,8 +421,9 @@ bool server_tma_applies(uint64_t n, uint64_t bucket)
 }
 
 // mode 1: dst = params (update with lr); mode 0: dst = acc (overwrite); mode 2: dst = acc (add into)
-cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
-                              float* params, float lr, int mode, cudaStream_t stream)
+template <bool RANGE>
+static cudaError_t launch_server_tma_codec(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                                           float* params, float lr, int mode, cudaStream_t stream)
 {
     ServerTmaArgs a;
     a.ptrs = ptrs;
@@ -437,16 +445,28 @@ cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
     unsigned int* timeouts = wait_timeout_counter();
     if (timeouts == nullptr) return cudaErrorNotSupported;
     switch (bits) {
-        case 1: return launch_server_tma_bits<1>(params, a, mode, timeouts, stream);
-        case 2: return launch_server_tma_bits<2>(params, a, mode, timeouts, stream);
-        case 3: return launch_server_tma_bits<3>(params, a, mode, timeouts, stream);
-        case 4: return launch_server_tma_bits<4>(params, a, mode, timeouts, stream);
-        case 5: return launch_server_tma_bits<5>(params, a, mode, timeouts, stream);
-        case 6: return launch_server_tma_bits<6>(params, a, mode, timeouts, stream);
-        case 7: return launch_server_tma_bits<7>(params, a, mode, timeouts, stream);
-        case 8: return launch_server_tma_bits<8>(params, a, mode, timeouts, stream);
+        case 1: return launch_server_tma_bits<1, RANGE>(params, a, mode, timeouts, stream);
+        case 2: return launch_server_tma_bits<2, RANGE>(params, a, mode, timeouts, stream);
+        case 3: return launch_server_tma_bits<3, RANGE>(params, a, mode, timeouts, stream);
+        case 4: return launch_server_tma_bits<4, RANGE>(params, a, mode, timeouts, stream);
+        case 5: return launch_server_tma_bits<5, RANGE>(params, a, mode, timeouts, stream);
+        case 6: return launch_server_tma_bits<6, RANGE>(params, a, mode, timeouts, stream);
+        case 7: return launch_server_tma_bits<7, RANGE>(params, a, mode, timeouts, stream);
+        case 8: return launch_server_tma_bits<8, RANGE>(params, a, mode, timeouts, stream);
     }
     return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                              float* params, float lr, int mode, cudaStream_t stream)
+{
+    return launch_server_tma_codec<false>(ptrs, W, bits, n, bucket, params, lr, mode, stream);
+}
+
+cudaError_t launch_server_range_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                                    float* params, float lr, int mode, cudaStream_t stream)
+{
+    return launch_server_tma_codec<true>(ptrs, W, bits, n, bucket, params, lr, mode, stream);
 }
 
 }  // namespace mqg
