@@ -487,6 +487,54 @@ def run_ours(args):
                                   "peak_kind": "148 SMs x 128 lanes x sampled SM clock",
                                   "ops_per_element": 4 * W + 13}}
 
+    # ---- codec variant (outside `value`): (min, max) range with nearest rounding, same workload, one
+    # launch per worker; bytes per element as the main codec plus 4 / B for the second float of a range
+    mm_ranges = [torch.zeros(2 * mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(W)]
+    mm_tab = (C.c_void_p * W)(*[t.data_ptr() for t in mm_ranges])
+    mm_steps = max(3, min(args.steps, 20))
+
+    def mm_quantize(b):
+        for w in range(W):
+            check(lib.mqg_quantize_minmax(grads[w].data_ptr(), n, b, B, codes[b][w].data_ptr(),
+                                          mm_ranges[w].data_ptr(), 0, sptr))
+
+    def mm_server(b):
+        check(lib.mqg_server_step_minmax(code_tab[b], mm_tab, W, b, n, B, params[b].data_ptr(), LR, None, sptr))
+
+    for b in ALL_BITS:
+        mm_quantize(b)
+    mm_events = []
+    for i in range(mm_steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(stream)
+        for b in ALL_BITS:
+            mm_quantize(b)
+        ev[1].record(stream)
+        for b in ALL_BITS:
+            mm_server(b)
+        ev[2].record(stream)
+        mm_events.append(ev)
+    torch.cuda.synchronize()
+    mm_q_s = float(np.mean([e[0].elapsed_time(e[1]) for e in mm_events])) * 1e-3
+    mm_s_s = float(np.mean([e[1].elapsed_time(e[2]) for e in mm_events])) * 1e-3
+    extra = 4 * mqg.mqg_num_buckets(n, B)
+    mm_q_bytes = sum(W * (quantize_bytes(n, b, B) + extra) for b in ALL_BITS)
+    mm_s_bytes = sum(server_bytes(n, b, B, W) + W * extra for b in ALL_BITS)
+    variant_minmax = {
+        "codec": "(min, max) range per bucket, nearest rounding (mqg_quantize_minmax / mqg_server_step_minmax); "
+                 "not part of `value`",
+        "quantize": {"avg_launch_us": mm_q_s / (len(ALL_BITS) * W) * 1e6, "launches_per_step": len(ALL_BITS) * W,
+                     "roofline": {"bound": "hbm", "achieved": mm_q_bytes / mm_q_s / 1e9, "peak": peak, "unit": "GB/s",
+                                  "frac": mm_q_bytes / mm_q_s / 1e9 / peak, "traffic": None}},
+        "server": {"avg_launch_us": mm_s_s / len(ALL_BITS) * 1e6, "launches_per_step": len(ALL_BITS),
+                   "roofline": {"bound": "hbm", "achieved": mm_s_bytes / mm_s_s / 1e9, "peak": peak, "unit": "GB/s",
+                                "frac": mm_s_bytes / mm_s_s / 1e9 / peak, "traffic": None}},
+    }
+    # put the codes back as the main codec writes them (the end-to-end leg re-quantizes anyway)
+    for b in ALL_BITS:
+        quantize_all(b, 0)
+    torch.cuda.synchronize()
+
     # ---- end to end from pinned host buffers
     e2e_steps = max(1, min(args.steps, 3))
     e2e_step(0)
@@ -515,6 +563,7 @@ def run_ours(args):
             "clocks": clocks.summary(), "e2e": e2e,
             "gpu_launches": args.steps * len(ALL_BITS) * (q_launches + 1),
             "roofline": roofline, "roofline_server": roofline_server, "downlink": downlink_line,
+            "variant_minmax": variant_minmax,
             "per_bits": per_bits,
         }
         if cpu is not None:
