@@ -23,6 +23,10 @@
  * The (min, max) nearest-rounding variant at the end of the file (readings M1..M4) is
  * pinned by exact rational arithmetic, dyadic closed forms, the half-step error bound,
  * monotonicity, end points and saturation.
+ * The L2-norm scale variant (readings N1..N3, after the (min, max) variant) is pinned by
+ * closed forms where every sum is exact, by inputs built so that another summation order or
+ * an unfused square gives another float, by exact rational arithmetic with one rounding per
+ * named operation, and by the error bound of its sum against the norm in double precision.
  * Parity unpinned: both codecs as a whole against the paper -- the paper prints no
  * worked example, error bound or sample output of Quantize / De-quantize.
  */
@@ -416,4 +420,94 @@ int mqo_server_step_minmax(const uint32_t *const *codes, const float *const *ran
     }
     free(acc);
     return rc;
+}
+
+/* ---- codec variant: L2-norm scale --------------------------------------------
+ * The paper's related-work section cites quantizers that scale by the Euclidean
+ * norm of the vector instead of its largest magnitude.  Only the scale differs
+ * from the main codec; the encode, the draws, the packing and the whole server
+ * side (R4..R14) are unchanged.  A sum of floats depends on its order, so the
+ * order is part of the definition (readings N1..N3):
+ *   N1  the bucket is cut into rows of 32 consecutive elements from its first
+ *       element (the last row may be shorter).  A row's sum of squares is the
+ *       left-to-right chain a <- fma(x_j, x_j, a), starting from a = 0.
+ *   N2  the row sums are the leaves of a balanced binary tree of adjacent pairs
+ *       (the leaf count padded with zeros to a power of two); each node is the
+ *       fp32 sum of its two children.  S = the root.
+ *   N3  S < 2^-96 flushes the bucket (scale 0, every code 0); otherwise the scale
+ *       is s = fl(sqrt(S)).  With that threshold every |x_i| <= s: a square that
+ *       is a normal number has an exact root, and smaller elements are below 2^-48.
+ * Inputs whose sum of squares overflows are outside the definition.
+ */
+float mqo_sumsq_tree(const float *x, uint64_t len)
+{
+    if (len == 0) return 0.0f;
+    uint64_t rows = (len + 31) / 32;
+    uint64_t padded = 1;
+    while (padded < rows) padded *= 2;
+    float *node = (float *)calloc(padded, sizeof(float));
+    if (!node) return NAN;
+    for (uint64_t r = 0; r < rows; ++r) {                 /* N1 */
+        uint64_t j0 = 32 * r, j1 = j0 + 32;
+        if (j1 > len) j1 = len;
+        float a = 0.0f;
+        for (uint64_t j = j0; j < j1; ++j) a = fmaf(x[j], x[j], a);
+        node[r] = a;
+    }
+    for (uint64_t width = padded; width > 1; width /= 2)  /* N2: one tree level per pass */
+        for (uint64_t j = 0; j < width / 2; ++j)
+            node[j] = node[2 * j] + node[2 * j + 1];
+    float S = node[0];
+    free(node);
+    return S;
+}
+
+void mqo_bucket_norms(const float *x, uint64_t n, uint64_t bucket, float *scales)
+{
+    const float tiny = ldexpf(1.0f, -96);
+    uint64_t nb = (n + bucket - 1) / bucket;
+    for (uint64_t k = 0; k < nb; ++k) {
+        uint64_t b0 = k * bucket, b1 = b0 + bucket;
+        if (b1 > n) b1 = n;
+        float S = mqo_sumsq_tree(x + b0, b1 - b0);
+        scales[k] = (S < tiny) ? 0.0f : sqrtf(S);         /* N3 */
+    }
+}
+
+/* Quantize(g, K) with the L2-norm scale: mqo_quantize with N1..N3 in place of R2/R3. */
+int mqo_quantize_l2(const void *grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                    uint32_t *codes, float *scales, int dtype, uint32_t worker,
+                    uint32_t step, uint64_t elem_offset)
+{
+    if (bits < 1 || bits > 8 || bucket == 0) return -1;
+    if (n == 0) return 0;
+    float *x = (float *)malloc(n * sizeof(float));
+    uint16_t *h = (uint16_t *)malloc(n * sizeof(uint16_t));
+    uint8_t *q = (uint8_t *)malloc(n);
+    if (!x || !h || !q) { free(x); free(h); free(q); return -2; }
+    if (dtype == 1) mqo_widen_bf16((const uint16_t *)grad, n, x);
+    else memcpy(x, grad, n * sizeof(float));
+    mqo_bucket_norms(x, n, bucket, scales);
+    mqo_draw_h(seed, worker, step, elem_offset, n, h);
+    mqo_encode(x, n, bits, bucket, scales, h, q);
+    mqo_pack(q, n, bits, codes);
+    free(x); free(h); free(q);
+    return 0;
+}
+
+/* Per-layer L2-norm scale: the segment conventions of mqo_quantize_segments. */
+int mqo_quantize_segments_l2(const void *grad, int nseg, const uint64_t *seg_off,
+                             const uint64_t *code_off, int bits, uint64_t seed,
+                             uint32_t *codes, float *scales, int dtype, uint32_t worker,
+                             uint32_t step, uint64_t elem_offset)
+{
+    for (int j = 0; j < nseg; ++j) {
+        uint64_t len = seg_off[j + 1] - seg_off[j];
+        const char *base = (const char *)grad + seg_off[j] * (dtype == 1 ? 2u : 4u);
+        if (len == 0) { scales[j] = 0.0f; continue; }
+        int rc = mqo_quantize_l2(base, len, bits, len, seed, codes + code_off[j], &scales[j],
+                                 dtype, worker, step, elem_offset + seg_off[j]);
+        if (rc) return rc;
+    }
+    return 0;
 }

@@ -286,3 +286,52 @@ def server_step_minmax(codes, ranges, bits, n, bucket, params, lr, want_acc=Fals
     if rc:
         raise ValueError("mqo_server_step_minmax failed: %d" % rc)
     return params, acc
+
+
+# ---- codec variant: L2-norm scale -----------------------------------------------------------
+_sumsq = _decl("mqo_sumsq_tree", C.c_float, _vp, _u64)
+_norms = _decl("mqo_bucket_norms", None, _vp, _u64, _u64, _vp)
+_quantize_l2 = _decl("mqo_quantize_l2", _int, _vp, _u64, _int, _u64, _u64, _vp, _vp, _int, _u32,
+                     _u32, _u64)
+_qseg_l2 = _decl("mqo_quantize_segments_l2", _int, _vp, _int, _vp, _vp, _int, _u64, _vp, _vp, _int,
+                 _u32, _u32, _u64)
+
+
+def sumsq_tree(x):
+    """The fixed-order fp32 sum of squares of one bucket (as a numpy float32)."""
+    x = _c(x, np.float32)
+    return np.float32(_sumsq(_ptr(x), x.size))
+
+
+def bucket_norms(x, bucket):
+    x = _c(x, np.float32)
+    s = np.empty(num_buckets(x.size, bucket), np.float32)
+    _norms(_ptr(x), x.size, bucket, _ptr(s))
+    return s
+
+
+def quantize_l2(grad, bits, bucket, seed, worker=0, step=0, elem_offset=0, dtype="f32"):
+    grad = _c(grad, np.uint16 if dtype == "bf16" else np.float32)
+    n = grad.size
+    codes = np.zeros(code_words(n, bits), np.uint32)
+    scales = np.zeros(num_buckets(n, bucket) if n else 0, np.float32)
+    rc = _quantize_l2(_ptr(grad), n, bits, bucket, seed, _ptr(codes), _ptr(scales),
+                      1 if dtype == "bf16" else 0, worker, step, elem_offset)
+    if rc:
+        raise ValueError("mqo_quantize_l2 failed: %d" % rc)
+    return codes, scales
+
+
+def quantize_segments_l2(grad, seg_off, code_off, bits, seed, worker=0, step=0, elem_offset=0,
+                         dtype="f32"):
+    grad = _c(grad, np.uint16 if dtype == "bf16" else np.float32)
+    seg_off = _c(seg_off, np.uint64)
+    code_off = _c(code_off, np.uint64)
+    nseg = seg_off.size - 1
+    codes = np.zeros(int(code_off[-1]), np.uint32)
+    scales = np.zeros(nseg, np.float32)
+    rc = _qseg_l2(_ptr(grad), nseg, _ptr(seg_off), _ptr(code_off), bits, seed, _ptr(codes),
+                  _ptr(scales), 1 if dtype == "bf16" else 0, worker, step, elem_offset)
+    if rc:
+        raise ValueError("mqo_quantize_segments_l2 failed: %d" % rc)
+    return codes, scales

@@ -1,5 +1,5 @@
 """Plants single mistakes in a copy of the CPU checker and verifies that the pin
-suites (tests/test_oracle_pins.py, tests/test_oracle_minmax_pins.py) reject every one of them.  Everything here runs
+suites (tests/test_oracle_pins.py, tests/test_oracle_minmax_pins.py, tests/test_oracle_l2_pins.py) reject every one of them.  Everything here runs
 on the CPU; the planted copies are compiled into a temporary directory."""
 import os
 import subprocess
@@ -62,6 +62,25 @@ MUTANTS_MINMAX = [
      "for (int w = 0; w < W - (W > 2); ++w) {\n        mqo_unpack(codes[w], n, bits, q);\n        mqo_dequantize_minmax"),
 ]
 
+# mistakes planted in the L2-norm scale variant, caught by tests/test_oracle_l2_pins.py
+MUTANTS_L2 = [
+    ("l2_rows_summed_in_sequence",
+     "for (uint64_t width = padded; width > 1; width /= 2)  /* N2: one tree level per pass */\n"
+     "        for (uint64_t j = 0; j < width / 2; ++j)\n"
+     "            node[j] = node[2 * j] + node[2 * j + 1];",
+     "for (uint64_t j = 1; j < padded; ++j) node[0] = node[0] + node[j];"),
+    ("l2_pairs_half_a_level_apart", "node[j] = node[2 * j] + node[2 * j + 1];", "node[j] = node[j] + node[j + width / 2];"),
+    ("l2_unfused_square", "a = fmaf(x[j], x[j], a);", "a = x[j] * x[j] + a;"),
+    ("l2_chain_right_to_left", "for (uint64_t j = j0; j < j1; ++j) a = fmaf(x[j], x[j], a);",
+     "for (uint64_t j = j1; j-- > j0; ) a = fmaf(x[j], x[j], a);"),
+    ("l2_short_last_row_dropped", "uint64_t rows = (len + 31) / 32;", "uint64_t rows = len >= 32 ? len / 32 : 1;"),
+    ("l2_rows_of_16", "uint64_t j0 = 32 * r, j1 = j0 + 32;", "uint64_t j0 = 32 * r, j1 = j0 + 16;"),
+    ("l2_no_root", "scales[k] = (S < tiny) ? 0.0f : sqrtf(S);", "scales[k] = (S < tiny) ? 0.0f : S;"),
+    ("l2_flush_decided_on_root", "scales[k] = (S < tiny) ? 0.0f : sqrtf(S);", "scales[k] = (sqrtf(S) < tiny) ? 0.0f : sqrtf(S);"),
+    ("l2_sum_of_magnitudes", "a = fmaf(x[j], x[j], a);", "a = fabsf(x[j]) + a;"),
+    ("l2_scale_is_max_abs", "mqo_bucket_norms(x, n, bucket, scales);\n    mqo_draw_h", "mqo_bucket_scales(x, n, bucket, scales);\n    mqo_draw_h"),
+]
+
 
 def _run(args):
     name, old, new, tmpdir = args
@@ -75,7 +94,8 @@ def _run(args):
     subprocess.run(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math", "-fPIC",
                     "-shared", "-o", so, c, "-lm"], check=True)
     env = dict(os.environ, MQG_ORACLE_LIB=so)
-    pins = "test_oracle_minmax_pins.py" if name.startswith("mm_") else "test_oracle_pins.py"
+    pins = ("test_oracle_minmax_pins.py" if name.startswith("mm_")
+            else "test_oracle_l2_pins.py" if name.startswith("l2_") else "test_oracle_pins.py")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         os.path.join(ROOT, "tests", pins)],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
@@ -83,7 +103,7 @@ def _run(args):
 
 
 def test_every_planted_mistake_is_caught(tmp_path):
-    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS + MUTANTS_MINMAX]
+    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS + MUTANTS_MINMAX + MUTANTS_L2]
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 2)) as ex:
         results = list(ex.map(_run, jobs))
     survivors = [name for name, rc, _ in results if rc == 0]
