@@ -171,6 +171,45 @@ mqg_status mqg_server_step_minmax(const uint32_t* const* codes, const float* con
                                   void* cuda_stream);
 
 /*
+ * Codec variant: the bucket's scale is its Euclidean norm, as in the norm-scaled quantizers the
+ * related-work section (Section 2) cites, instead of its largest magnitude.  Everything else is
+ * mqg_quantize: same encode against [-s, +s], same draws, same packing, and the outputs are
+ * consumed by the ordinary server calls (mqg_server_step, mqg_dequant_accumulate,
+ * mqg_server_requantize).  Because a float sum depends on its order, the order is fixed:
+ *   - the bucket is cut into rows of 32 consecutive elements from its first element; a row's sum
+ *     of squares is the chain a <- fma(x_j, x_j, a), left to right, from a = 0;
+ *   - the row sums are combined by a balanced binary tree of adjacent pairs (leaf count padded
+ *     with zeros to a power of two); S is the root;
+ *   - scales[k] = 0 if S < 2^-96 (every code of the bucket is then 0), else sqrt(S) rounded once.
+ * The result is therefore reproducible bit for bit, on any device and launch shape.  Inputs whose
+ * sum of squares overflows fp32 give unspecified results.
+ * Buckets (or a single bucket n) above 8192 elements are rejected with MQG_ERR_INVALID: use the
+ * segment form below for those.  Other arguments and errors as mqg_quantize.
+ */
+mqg_status mqg_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                           uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                           uint32_t step, uint64_t elem_offset, void* cuda_stream);
+
+/*
+ * The same variant with one norm per segment (per-layer scale), segment tables as in
+ * mqg_quantize_segments below; the outputs go to mqg_server_step_segments.  The rows and the
+ * tree of a segment start at the segment's first element.
+ *   workspace        [scratch] DEVICE memory for the partial sums: at least
+ *                    mqg_l2_workspace_floats(nseg, seg_off) floats (one per 8192 elements of every
+ *                    segment, rounded up per segment), 4-byte aligned.  Contents on entry do not
+ *                    matter and are undefined on return; calls that may run concurrently on the
+ *                    device need separate workspaces.
+ *   workspace_floats its size in floats; MQG_ERR_INVALID when too small.
+ * The gradient is read twice (sum pass, encode pass).
+ */
+size_t mqg_l2_workspace_floats(int nseg, const uint64_t* seg_off);
+mqg_status mqg_quantize_segments_l2(const void* grad, int nseg, const uint64_t* seg_off,
+                                    const uint64_t* code_off, int bits, uint64_t seed,
+                                    uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                                    uint32_t step, uint64_t elem_offset, float* workspace,
+                                    size_t workspace_floats, void* cuda_stream);
+
+/*
  * Per-layer scale ("gradient quantization is applied to these two layers", Section 4.1): the flat
  * gradient is cut into nseg segments; segment j = elements [seg_off[j], seg_off[j+1]) is ONE bucket
  * with scale scales[j], and its bit stream starts on a word boundary at word code_off[j].

@@ -8,7 +8,8 @@ raises.
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_quantize_minmax,
-  mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_code_words, mqg_num_buckets,
+  mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_segments_l2,
+  mqg_l2_workspace_floats, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
 from __future__ import annotations
@@ -60,6 +61,10 @@ def _load() -> C.CDLL:
         "mqg_server_requantize": (i32, [vp, vp, i32, i32, u64, u64, f32, u64, vp, vp, u32, u32, vp]),
         "mqg_quantize_segments": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_server_step_segments": (i32, [vp, vp, i32, i32, i32, vp, vp, vp, f32, vp, vp]),
+        "mqg_quantize_l2": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
+        "mqg_l2_workspace_floats": (C.c_size_t, [i32, vp]),
+        "mqg_quantize_segments_l2": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp,
+                                           C.c_size_t, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -228,6 +233,28 @@ def mqg_server_step_segments(codes, scales, W: int, bits: int, seg_off, code_off
                                          _dev_ptr(params, "params"), lr,
                                          _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
                                          _stream()))
+
+
+def mqg_quantize_l2(grad, n: int, bits: int, bucket: int, seed: int, codes, scales,
+                    worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    _check(_lib.mqg_quantize_l2(_dev_ptr(grad, "grad"), n, bits, bucket, seed & 0xFFFFFFFFFFFFFFFF,
+                                _dev_ptr(codes, "codes"), _dev_ptr(scales, "scales"),
+                                _grad_dtype(grad), worker, step, elem_offset, _stream()))
+
+
+def mqg_l2_workspace_floats(seg_off) -> int:
+    return int(_lib.mqg_l2_workspace_floats(len(seg_off) - 1, _u64_table(seg_off)))
+
+
+def mqg_quantize_segments_l2(grad, seg_off, code_off, bits: int, seed: int, codes, scales, workspace,
+                             worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    """`workspace`: float32 CUDA tensor of at least mqg_l2_workspace_floats(seg_off) elements."""
+    nseg = len(seg_off) - 1
+    _check(_lib.mqg_quantize_segments_l2(_dev_ptr(grad, "grad"), nseg, _u64_table(seg_off),
+                                         _u64_table(code_off), bits, seed & 0xFFFFFFFFFFFFFFFF,
+                                         _dev_ptr(codes, "codes"), _dev_ptr(scales, "scales"),
+                                         _grad_dtype(grad), worker, step, elem_offset,
+                                         _dev_ptr(workspace, "workspace"), workspace.numel(), _stream()))
 
 
 def raw_library() -> C.CDLL:

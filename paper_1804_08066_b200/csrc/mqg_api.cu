@@ -359,6 +359,73 @@ mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg
         });
 }
 
+mqg_status mqg_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                           uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                           uint32_t step, uint64_t elem_offset, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (n == 0) return MQG_OK;
+    if ((bucket < n ? bucket : n) > (uint64_t)mqg::kMaxFusedBucket)
+        return fail(MQG_ERR_INVALID, "mqg_quantize_l2 supports buckets of at most %d elements; use "
+                    "mqg_quantize_segments_l2 for longer ones", mqg::kMaxFusedBucket);
+    if (!grad || !codes || !scales) return fail(MQG_ERR_INVALID, "grad, codes or scales is null");
+    if (!aligned16(grad)) return fail(MQG_ERR_ALIGN, "grad not 16-byte aligned");
+    if (!aligned16(codes)) return fail(MQG_ERR_ALIGN, "codes not 16-byte aligned");
+    if (!aligned4(scales)) return fail(MQG_ERR_ALIGN, "scales not 4-byte aligned");
+    const cudaError_t err = mqg::launch_quantize_l2(grad, n, bits, bucket, seed, codes, scales, (int)dtype,
+                                                    worker, step, elem_offset,
+                                                    static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_quantize_l2", err);
+    return MQG_OK;
+}
+
+size_t mqg_l2_workspace_floats(int nseg, const uint64_t* seg_off)
+{
+    if (nseg <= 0 || !seg_off) return 0;
+    const uint64_t tile_elems = (uint64_t)mqg::kMaxTileRows * 32;
+    uint64_t tiles = 0;
+    for (int j = 0; j < nseg; ++j)
+        if (seg_off[j + 1] > seg_off[j]) tiles += (seg_off[j + 1] - seg_off[j] + tile_elems - 1) / tile_elems;
+    return (size_t)tiles;
+}
+
+mqg_status mqg_quantize_segments_l2(const void* grad, int nseg, const uint64_t* seg_off,
+                                    const uint64_t* code_off, int bits, uint64_t seed,
+                                    uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
+                                    uint32_t step, uint64_t elem_offset, float* workspace,
+                                    size_t workspace_floats, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (nseg > 0) {
+        if (!grad || !codes || !scales) return fail(MQG_ERR_INVALID, "grad, codes or scales is null");
+        if (!aligned16(grad)) return fail(MQG_ERR_ALIGN, "grad not 16-byte aligned");
+        if (!aligned16(codes)) return fail(MQG_ERR_ALIGN, "codes not 16-byte aligned");
+        if (!aligned4(scales)) return fail(MQG_ERR_ALIGN, "scales not 4-byte aligned");
+        if (!seg_off || !code_off) return fail(MQG_ERR_INVALID, "segment table is null");
+        const size_t need = mqg_l2_workspace_floats(nseg, seg_off);
+        if (need > workspace_floats)
+            return fail(MQG_ERR_INVALID, "workspace holds %llu floats, %llu needed (mqg_l2_workspace_floats)",
+                        (unsigned long long)workspace_floats, (unsigned long long)need);
+        if (need != 0 && !workspace) return fail(MQG_ERR_INVALID, "workspace is null");
+        if (!aligned4(workspace)) return fail(MQG_ERR_ALIGN, "workspace not 4-byte aligned");
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    size_t used = 0;                      // tiles of the chunks already launched
+    return for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            const cudaError_t err = mqg::launch_quantize_segments_l2(grad, tab, bits, seed, codes,
+                                                                     scales + first, (int)dtype, worker,
+                                                                     step, elem_offset, workspace + used,
+                                                                     stream);
+            if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_l2", err);
+            used += tab.tile_start[tab.nseg];
+            return MQG_OK;
+        });
+}
+
 mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* const* scales, int W,
                                     int bits, int nseg, const uint64_t* seg_off,
                                     const uint64_t* code_off, float* params, float lr,

@@ -62,6 +62,17 @@ cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, 
                                      uint32_t worker, uint32_t step, uint64_t elem_offset,
                                      cudaStream_t stream);
 
+// L2-norm scale variant.  Buckets of at most kMaxFusedBucket elements: one pass.  Segments: tile
+// sums into `partial` (one float per tile of the table, in tile order), a fold per segment, then
+// the ordinary encode pass.
+cudaError_t launch_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                               uint32_t* codes, float* scales, int dtype, uint32_t worker, uint32_t step,
+                               uint64_t elem_offset, cudaStream_t stream);
+cudaError_t launch_quantize_segments_l2(const void* grad, const SegmentTable& tab, int bits, uint64_t seed,
+                                        uint32_t* codes, float* scales_base, int dtype, uint32_t worker,
+                                        uint32_t step, uint64_t elem_offset, float* partial,
+                                        cudaStream_t stream);
+
 // Two-pass quantize with uniform large buckets (bucket > kMaxFusedBucket, or a single bucket
 // whose length is not a multiple of 32).
 cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, uint64_t bucket,

@@ -6,14 +6,6 @@
 
 namespace mqg {
 
-struct SegQuantArgs {
-    const void* grad;
-    uint32_t* codes;
-    float* scales;          // scale of segment j at scales[j]
-    uint64_t elem_offset;
-    DrawKey key;
-};
-
 template <int DTYPE>
 __global__ void __launch_bounds__(kMaxTileRows)
 absmax_segments_kernel(const SegQuantArgs a, const SegmentTable tab)
@@ -116,6 +108,22 @@ static cudaError_t launch_encode_bits(const SegQuantArgs& a, const SegmentTable&
     return cudaGetLastError();
 }
 
+cudaError_t launch_encode_segments(const SegQuantArgs& a, const SegmentTable& tab, int bits, int dtype,
+                                   unsigned grid, cudaStream_t stream)
+{
+    switch (bits) {
+        case 1: return launch_encode_bits<1>(a, tab, dtype, grid, stream);
+        case 2: return launch_encode_bits<2>(a, tab, dtype, grid, stream);
+        case 3: return launch_encode_bits<3>(a, tab, dtype, grid, stream);
+        case 4: return launch_encode_bits<4>(a, tab, dtype, grid, stream);
+        case 5: return launch_encode_bits<5>(a, tab, dtype, grid, stream);
+        case 6: return launch_encode_bits<6>(a, tab, dtype, grid, stream);
+        case 7: return launch_encode_bits<7>(a, tab, dtype, grid, stream);
+        case 8: return launch_encode_bits<8>(a, tab, dtype, grid, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
 static cudaError_t two_pass(const SegQuantArgs& a, const SegmentTable& tab, uint64_t ntiles,
                             uint64_t nscales, int bits, int dtype, cudaStream_t stream)
 {
@@ -128,17 +136,7 @@ static cudaError_t two_pass(const SegQuantArgs& a, const SegmentTable& tab, uint
     else absmax_segments_kernel<1><<<grid, kMaxTileRows, 0, stream>>>(a, tab);
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    switch (bits) {
-        case 1: return launch_encode_bits<1>(a, tab, dtype, grid, stream);
-        case 2: return launch_encode_bits<2>(a, tab, dtype, grid, stream);
-        case 3: return launch_encode_bits<3>(a, tab, dtype, grid, stream);
-        case 4: return launch_encode_bits<4>(a, tab, dtype, grid, stream);
-        case 5: return launch_encode_bits<5>(a, tab, dtype, grid, stream);
-        case 6: return launch_encode_bits<6>(a, tab, dtype, grid, stream);
-        case 7: return launch_encode_bits<7>(a, tab, dtype, grid, stream);
-        case 8: return launch_encode_bits<8>(a, tab, dtype, grid, stream);
-    }
-    return cudaErrorInvalidValue;
+    return launch_encode_segments(a, tab, bits, dtype, grid, stream);
 }
 
 cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, int bits,

@@ -7,6 +7,19 @@
 
 namespace mqg {
 
+struct SegQuantArgs {
+    const void* grad;
+    uint32_t* codes;
+    float* scales;          // scale of segment j at scales[j]
+    uint64_t elem_offset;
+    DrawKey key;
+};
+
+// The encode pass of the segment quantizers: one CTA per tile, scale of the tile's segment read
+// from a.scales (already final, or the raw maximum that the first tile then flushes).
+cudaError_t launch_encode_segments(const SegQuantArgs& a, const SegmentTable& tab, int bits, int dtype,
+                                   unsigned grid, cudaStream_t stream);
+
 struct TileGeom {
     uint64_t elem0;       // flat index of the tile's first element
     uint64_t valid;       // elements from elem0 to the end of the segment
