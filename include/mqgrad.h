@@ -210,6 +210,36 @@ mqg_status mqg_quantize_segments_l2(const void* grad, int nseg, const uint64_t* 
                                     size_t workspace_floats, void* cuda_stream);
 
 /*
+ * mqg_quantize_segments_l2 without the workspace argument, for callers that cannot supply device
+ * memory of their own: processes whose device memory has all been handed to one pool at start-up
+ * (a later allocation fails), latency-critical paths that must not run into the device-wide
+ * synchronisation of an allocation, and plug-ins or callbacks whose host only lets them launch
+ * work on the buffers they are given.  (The paper has no counterpart: this is a property of the
+ * library's interface, not of the method.)  The partial sums go to an array inside the library
+ * image instead; arguments, results and errors are otherwise exactly those of
+ * mqg_quantize_segments_l2.
+ *   - Limit: mqg_l2_workspace_floats(nseg, seg_off) <= MQG_L2_STATIC_WORKSPACE_FLOATS (65,536 partial
+ *     sums, one per started 8192 elements of every segment: about 5 * 10^8 elements); beyond it the
+ *     call returns MQG_ERR_INVALID, enqueues nothing, and mqg_last_error() names both numbers.
+ *   - Cost: the array (256 KiB) occupies device memory on every GPU that loads the library, from
+ *     load until the process exits, also if this function is never called.
+ *   - The call allocates and frees nothing, on the host or the device.  The first call on each
+ *     device looks up the array's device address (once; later calls reuse it); make that first
+ *     call before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps what the last call left in it.
+ *     Nothing in it needs to be zero on entry (every element read is written earlier in the same
+ *     call), but two calls whose kernels can overlap on the device - different streams, or
+ *     different host threads on different streams - race on it and corrupt each other's scales:
+ *     order them on one stream or with events.
+ */
+#define MQG_L2_STATIC_WORKSPACE_FLOATS 65536
+mqg_status mqg_quantize_segments_l2_static(const void* grad, int nseg, const uint64_t* seg_off,
+                                           const uint64_t* code_off, int bits, uint64_t seed,
+                                           uint32_t* codes, float* scales, mqg_dtype dtype,
+                                           uint32_t worker, uint32_t step, uint64_t elem_offset,
+                                           void* cuda_stream);
+
+/*
  * Per-layer scale ("gradient quantization is applied to these two layers", Section 4.1): the flat
  * gradient is cut into nseg segments; segment j = elements [seg_off[j], seg_off[j+1]) is ONE bucket
  * with scale scales[j], and its bit stream starts on a word boundary at word code_off[j].

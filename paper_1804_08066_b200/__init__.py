@@ -9,7 +9,7 @@ Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_quantize_minmax,
   mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_segments_l2,
-  mqg_l2_workspace_floats, mqg_code_words, mqg_num_buckets,
+  mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
 from __future__ import annotations
@@ -65,6 +65,7 @@ def _load() -> C.CDLL:
         "mqg_l2_workspace_floats": (C.c_size_t, [i32, vp]),
         "mqg_quantize_segments_l2": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp,
                                            C.c_size_t, vp]),
+        "mqg_quantize_segments_l2_static": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -255,6 +256,21 @@ def mqg_quantize_segments_l2(grad, seg_off, code_off, bits: int, seed: int, code
                                          _dev_ptr(codes, "codes"), _dev_ptr(scales, "scales"),
                                          _grad_dtype(grad), worker, step, elem_offset,
                                          _dev_ptr(workspace, "workspace"), workspace.numel(), _stream()))
+
+
+MQG_L2_STATIC_WORKSPACE_FLOATS = 65536
+
+
+def mqg_quantize_segments_l2_static(grad, seg_off, code_off, bits: int, seed: int, codes, scales,
+                                    worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    """mqg_quantize_segments_l2 for callers that cannot supply a workspace: the partial sums use an
+    array inside the library (at most MQG_L2_STATIC_WORKSPACE_FLOATS of them); calls that may
+    overlap on the device must be ordered by the caller."""
+    nseg = len(seg_off) - 1
+    _check(_lib.mqg_quantize_segments_l2_static(_dev_ptr(grad, "grad"), nseg, _u64_table(seg_off),
+                                                _u64_table(code_off), bits, seed & 0xFFFFFFFFFFFFFFFF,
+                                                _dev_ptr(codes, "codes"), _dev_ptr(scales, "scales"),
+                                                _grad_dtype(grad), worker, step, elem_offset, _stream()))
 
 
 def raw_library() -> C.CDLL:

@@ -112,6 +112,15 @@ mqg_status for_each_chunk(int nseg, const uint64_t* seg_off, const uint64_t* cod
 
 }  // namespace
 
+int mqg::report_error(int code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
 extern "C" {
 
 size_t mqg_code_words(uint64_t n, int bits) { return (size_t)((n * (uint64_t)bits + 31) / 32); }

@@ -6,6 +6,10 @@
 
 namespace mqg {
 
+// For entry points implemented outside mqg_api.cu: stores the calling thread's message for
+// mqg_last_error() and returns `code`.
+int report_error(int code, const char* fmt, ...);
+
 constexpr int kMaxWorkers = 32;
 constexpr int kMaxSegmentsPerLaunch = 64;
 
