@@ -530,6 +530,31 @@ def run_ours(args):
                    "roofline": {"bound": "hbm", "achieved": mm_s_bytes / mm_s_s / 1e9, "peak": peak, "unit": "GB/s",
                                 "frac": mm_s_bytes / mm_s_s / 1e9 / peak, "traffic": None}},
     }
+    # ---- codec variant (outside `value`): L2-norm scale; only the quantizer differs (one launch per
+    # worker, bytes per element as the main codec), the server step is the main codec's
+    def l2_quantize(b, step_no):
+        for w in range(W):
+            check(lib.mqg_quantize_l2(grads[w].data_ptr(), n, b, B, PHILOX_SEED, codes[b][w].data_ptr(),
+                                      scales[b][w].data_ptr(), 0, w, step_no, 0, sptr))
+
+    for b in ALL_BITS:
+        l2_quantize(b, 0)
+    l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0.record(stream)
+    for i in range(mm_steps):
+        for b in ALL_BITS:
+            l2_quantize(b, 1 + i)
+    l1.record(stream)
+    torch.cuda.synchronize()
+    l2_q_s = l0.elapsed_time(l1) * 1e-3 / mm_steps
+    l2_q_bytes = sum(W * quantize_bytes(n, b, B) for b in ALL_BITS)
+    variant_l2 = {
+        "codec": "L2-norm scale per bucket, fixed summation tree (mqg_quantize_l2; server step as the main "
+                 "codec); not part of `value`",
+        "quantize": {"avg_launch_us": l2_q_s / (len(ALL_BITS) * W) * 1e6, "launches_per_step": len(ALL_BITS) * W,
+                     "roofline": {"bound": "hbm", "achieved": l2_q_bytes / l2_q_s / 1e9, "peak": peak, "unit": "GB/s",
+                                  "frac": l2_q_bytes / l2_q_s / 1e9 / peak, "traffic": None}},
+    }
     # put the codes back as the main codec writes them (the end-to-end leg re-quantizes anyway)
     for b in ALL_BITS:
         quantize_all(b, 0)
@@ -563,7 +588,7 @@ def run_ours(args):
             "clocks": clocks.summary(), "e2e": e2e,
             "gpu_launches": args.steps * len(ALL_BITS) * (q_launches + 1),
             "roofline": roofline, "roofline_server": roofline_server, "downlink": downlink_line,
-            "variant_minmax": variant_minmax,
+            "variant_minmax": variant_minmax, "variant_l2": variant_l2,
             "per_bits": per_bits,
         }
         if cpu is not None:

@@ -127,6 +127,16 @@ __device__ __forceinline__ float row_abs_max(const float (&x)[32])
     return mx;
 }
 
+// L2-norm scale variant: a row's sum of squares is the left-to-right chain a <- fma(x_j, x_j, a)
+// from a = 0 (the order is part of the variant's definition).
+__device__ __forceinline__ float row_sum_squares(const float (&x)[32])
+{
+    float a = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) a = __fmaf_rn(x[j], x[j], a);
+    return a;
+}
+
 // Per-bucket encode constants, pre-scaled by 2^16: T = fma(x, inv16, half_l16) = 2^16 * t with
 // t = fl(x * fl(L / 2s) + L/2) -- scaling both constants by a power of two leaves the single
 // rounding of the fma unchanged.  A flushed bucket uses (0, 0): every x gives T = 0, code 0.

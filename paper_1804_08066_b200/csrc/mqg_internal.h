@@ -69,6 +69,10 @@ cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, 
 // L2-norm scale variant.  Buckets of at most kMaxFusedBucket elements: one pass.  Segments: tile
 // sums into `partial` (one float per tile of the table, in tile order), a fold per segment, then
 // the ordinary encode pass.
+bool quantize_norm_fused_applies(uint64_t n, uint64_t bucket, uint64_t elem_offset);
+cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                                       uint32_t* codes, float* scales, int dtype, uint32_t worker,
+                                       uint32_t step, uint64_t elem_offset, cudaStream_t stream);
 cudaError_t launch_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
                                uint32_t* codes, float* scales, int dtype, uint32_t worker, uint32_t step,
                                uint64_t elem_offset, cudaStream_t stream);

@@ -16,14 +16,6 @@ namespace mqg {
 
 namespace {
 
-__device__ __forceinline__ float row_sum_squares(const float (&x)[32])
-{
-    float a = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) a = __fmaf_rn(x[j], x[j], a);
-    return a;
-}
-
 // Five tree levels inside a warp: lane l holds the sum of rows (l & ~(2d - 1)) .. + 2d - 1 after
 // the step with distance d.  Both partners compute the same sum (addition commutes bit for bit).
 __device__ __forceinline__ float warp_tree(float a, uint32_t levels_end)
@@ -226,6 +218,9 @@ cudaError_t launch_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t 
                                uint32_t* codes, float* scales, int dtype, uint32_t worker, uint32_t step,
                                uint64_t elem_offset, cudaStream_t stream)
 {
+    if (quantize_norm_fused_applies(n, bucket, elem_offset))        // TMA-fed persistent kernel
+        return launch_quantize_norm_fused(grad, n, bits, bucket, seed, codes, scales, dtype, worker, step,
+                                          elem_offset, stream);
     L2Args a;
     a.grad = grad; a.codes = codes; a.scales = scales;
     a.n = n;

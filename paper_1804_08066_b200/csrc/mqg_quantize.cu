@@ -201,7 +201,7 @@ struct WorkerView {
 // (lane shuffles); otherwise a whole number of warps (one shared-memory atomic per warp).  After
 // the tile's rows are in registers thread 0 calls `refill(stage, bar)` to start the copy that
 // uses the stage next.  Returns false if the tile's copy never landed.
-template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, typename Refill>
+template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, bool NORM = false, typename Refill>
 __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
                                               const QuantizeArgs& a, const TmaQuantizeConsts& c,
                                               uint32_t k, uint32_t tile, Refill&& refill,
@@ -227,25 +227,49 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
 #pragma unroll
         for (int j = 0; j < 32; ++j) x[j] = 0.0f;
     }
-    uint32_t m = __float_as_uint(row_abs_max(x));
+    uint32_t m;
     uint32_t* slot = sh.slots[k % 3];
-    if (SHUFFLE) {
-        for (uint32_t d = a.rows_per_bucket >> 1; d > 0; d >>= 1)
-            m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+    if constexpr (NORM) {
+        // L2-norm scale: the fixed tree over the rows' sums of squares - partner distance 1, 2, 4, ...
+        // inside the warp, then (buckets of whole warps) the warp sums, one slot per warp
+        float ss = row_sum_squares(x);
+        const uint32_t lanes = SHUFFLE ? a.rows_per_bucket : 32u;
+        for (uint32_t d = 1; d < lanes; d <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xFFFFFFFFu, ss, d));
+        if (!SHUFFLE && (t & 31) == 0) slot[t >> 5] = __float_as_uint(ss);
+        m = __float_as_uint(ss);
     } else {
-        m = __reduce_max_sync(0xFFFFFFFFu, m);
-        if ((t & 31) == 0) atomicMax(&slot[local_bucket], m);
+        m = __float_as_uint(row_abs_max(x));
+        if (SHUFFLE) {
+            for (uint32_t d = a.rows_per_bucket >> 1; d > 0; d >>= 1)
+                m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+        } else {
+            m = __reduce_max_sync(0xFFFFFFFFu, m);
+            if ((t & 31) == 0) atomicMax(&slot[local_bucket], m);
+        }
     }
     if (__syncthreads_or(!ok)) return false;
     if (t == 0) refill(smem_u32(stage), bar);                    // every thread has read the stage
     if (!SHUFFLE) {
-        m = slot[local_bucket];
-        if (t < THREADS / 32) sh.slots[(k + 2) % 3][t] = 0u;     // next used by this CTA's tile k + 2
+        if constexpr (NORM) {
+            // tree over the bucket's warp sums, zero leaves up to four (plain stores: nothing to reset;
+            // the slot array is written again two barriers from here)
+            static_assert(THREADS / 32 == 4, "the warp-sum tree is written for four warps");
+            const uint32_t wpb = a.rows_per_bucket >> 5, first = local_bucket * wpb;
+            float v[4];
+#pragma unroll
+            for (uint32_t i = 0; i < 4; ++i)
+                v[i] = (i < wpb && first + i < 4u) ? __uint_as_float(slot[first + i]) : 0.0f;
+            m = __float_as_uint(__fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3])));
+        } else {
+            m = slot[local_bucket];
+            if (t < THREADS / 32) sh.slots[(k + 2) % 3][t] = 0u; // next used by this CTA's tile k + 2
+        }
     }
     if (!active) return true;
 
     float sc = __uint_as_float(m);
-    if (sc < flush_limit()) sc = 0.0f;
+    if constexpr (NORM) sc = sc < flush_limit() ? 0.0f : __fsqrt_rn(sc);     // flush decided on the sum
+    else if (sc < flush_limit()) sc = 0.0f;
     const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
     if (scale_writer && (FULL || bucket < a.nbuckets)) wv.scales[bucket] = sc;
 
@@ -351,7 +375,10 @@ __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THR
     return true;
 }
 
-template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, bool RANGE = false>
+// MODE: kMaxAbs = the main codec, kRange = the (min, max) variant, kNorm = the L2-norm scale variant.
+enum : int { kMaxAbs = 0, kRange = 1, kNorm = 2 };
+
+template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, int MODE = kMaxAbs>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ QuantizeArgs a,
                     const __grid_constant__ TmaQuantizeConsts c, unsigned int* __restrict__ timeouts)
@@ -399,7 +426,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
                 tma_load_2d(stage, &tmap, 0, (int)(next_tile * a.tile_rows), bar);
             }
         };
-        if constexpr (RANGE) {
+        if constexpr (MODE == kRange) {
             if (tile < c.full_tiles)
                 ok = range_quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, k, tile, refill,
                                                                                local_bucket, scale_writer);
@@ -407,12 +434,13 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
                 ok = range_quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, k, tile, refill,
                                                                                 local_bucket, scale_writer);
         } else {
+            constexpr bool NORM = MODE == kNorm;
             if (tile < c.full_tiles)
-                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, tile, refill,
-                                                                         local_bucket, scale_writer);
+                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM>(sh, wv, a, c, k, tile, refill,
+                                                                               local_bucket, scale_writer);
             else
-                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, tile, refill,
-                                                                          local_bucket, scale_writer);
+                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM>(sh, wv, a, c, k, tile, refill,
+                                                                                local_bucket, scale_writer);
         }
     }
     if (!ok) {
@@ -523,12 +551,12 @@ static cudaError_t launch_bits(const QuantizeArgs& a, int dtype, bool aligned, u
     return cudaGetLastError();
 }
 
-template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, bool RANGE = false>
+template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, int MODE = kMaxAbs>
 static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a,
                                    const TmaQuantizeConsts& c, unsigned int* timeouts,
                                    cudaStream_t stream)
 {
-    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, SHUFFLE, RANGE>;
+    auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, SHUFFLE, MODE>;
     static int grid_cap[64] = {};                  // per device; 0 = not yet queried
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -753,10 +781,10 @@ static cudaError_t launch_range_bits(const CUtensorMap& map, const QuantizeArgs&
                                      int dtype, bool shuffle, unsigned int* timeouts, cudaStream_t stream)
 {
     if (dtype == 0)
-        return shuffle ? launch_tma_inst<BITS, 0, 128, true, true>(map, a, c, timeouts, stream)
-                       : launch_tma_inst<BITS, 0, 128, false, true>(map, a, c, timeouts, stream);
-    return shuffle ? launch_tma_inst<BITS, 1, 128, true, true>(map, a, c, timeouts, stream)
-                   : launch_tma_inst<BITS, 1, 128, false, true>(map, a, c, timeouts, stream);
+        return shuffle ? launch_tma_inst<BITS, 0, 128, true, kRange>(map, a, c, timeouts, stream)
+                       : launch_tma_inst<BITS, 0, 128, false, kRange>(map, a, c, timeouts, stream);
+    return shuffle ? launch_tma_inst<BITS, 1, 128, true, kRange>(map, a, c, timeouts, stream)
+                   : launch_tma_inst<BITS, 1, 128, false, kRange>(map, a, c, timeouts, stream);
 }
 
 bool quantize_range_fused_applies(uint64_t n, uint64_t bucket)
@@ -790,6 +818,54 @@ cudaError_t launch_quantize_range_fused(const void* grad, uint64_t n, int bits, 
         case 6: return launch_range_bits<6>(map, a, c, dtype, shuffle, timeouts, stream);
         case 7: return launch_range_bits<7>(map, a, c, dtype, shuffle, timeouts, stream);
         case 8: return launch_range_bits<8>(map, a, c, dtype, shuffle, timeouts, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// ---- L2-norm scale variant on the TMA kernel (buckets of at most 128 rows, block-aligned draws) ----
+template <int BITS>
+static cudaError_t launch_norm_bits(const CUtensorMap& map, const QuantizeArgs& a, const TmaQuantizeConsts& c,
+                                    int dtype, bool shuffle, unsigned int* timeouts, cudaStream_t stream)
+{
+    if (dtype == 0)
+        return shuffle ? launch_tma_inst<BITS, 0, 128, true, kNorm>(map, a, c, timeouts, stream)
+                       : launch_tma_inst<BITS, 0, 128, false, kNorm>(map, a, c, timeouts, stream);
+    return shuffle ? launch_tma_inst<BITS, 1, 128, true, kNorm>(map, a, c, timeouts, stream)
+                   : launch_tma_inst<BITS, 1, 128, false, kNorm>(map, a, c, timeouts, stream);
+}
+
+bool quantize_norm_fused_applies(uint64_t n, uint64_t bucket, uint64_t elem_offset)
+{
+    if (n == 0) return false;
+    const uint64_t nrows = (n + 31) / 32;
+    const uint64_t rpb = (bucket >= n) ? nrows : bucket / 32;
+    return tma_path_applies(n, rpb, elem_offset) && rpb <= 128;
+}
+
+cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
+                                       uint32_t* codes, float* scales, int dtype, uint32_t worker,
+                                       uint32_t step, uint64_t elem_offset, cudaStream_t stream)
+{
+    QuantizeArgs a;
+    const uint64_t rpb = fill_args(a, grad, n, bits, bucket, seed, codes, scales, worker, step, elem_offset);
+    TmaQuantizeConsts c;
+    if (fill_tma_args(a, c, rpb) != 128) return cudaErrorInvalidValue;
+    unsigned int* timeouts = wait_timeout_counter();
+    if (timeouts == nullptr) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const char* why = nullptr;
+    if (!encode_rows_map(&map, grad, a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why))
+        return cudaErrorNotSupported;
+    const bool shuffle = rpb <= 32;
+    switch (bits) {
+        case 1: return launch_norm_bits<1>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 2: return launch_norm_bits<2>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 3: return launch_norm_bits<3>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 4: return launch_norm_bits<4>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 5: return launch_norm_bits<5>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 6: return launch_norm_bits<6>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 7: return launch_norm_bits<7>(map, a, c, dtype, shuffle, timeouts, stream);
+        case 8: return launch_norm_bits<8>(map, a, c, dtype, shuffle, timeouts, stream);
     }
     return cudaErrorInvalidValue;
 }
