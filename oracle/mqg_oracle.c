@@ -27,6 +27,10 @@
  * closed forms where every sum is exact, by inputs built so that another summation order or
  * an unfused square gives another float, by exact rational arithmetic with one rounding per
  * named operation, and by the error bound of its sum against the norm in double precision.
+ * The 1-bit error-feedback variant (readings E1..E5, last in the file) is pinned by hand-
+ * computed small cases, by the conservation law sent + residual = gradient + old residual on
+ * exactly representable data, by numpy means on integer data, by order-sensitive inputs and
+ * by the separately pinned (min, max) de-quantizer as its receiver.
  * Parity unpinned: both codecs as a whole against the paper -- the paper prints no
  * worked example, error bound or sample output of Quantize / De-quantize.
  */
@@ -509,5 +513,91 @@ int mqo_quantize_segments_l2(const void *grad, int nseg, const uint64_t *seg_off
                                  dtype, worker, step, elem_offset + seg_off[j]);
         if (rc) return rc;
     }
+    return 0;
+}
+
+/* ---- codec variant: one bit per element with error feedback ---------------------
+ * Section 2 (Related work) cites the 1-bit scheme in which every gradient value travels
+ * as one bit and the quantization error is carried forward into the next mini-batch.
+ * The paper gives no formula for it; the readings this repository fixes (E1..E5):
+ *   E1  v_i = fl(g_i + e_i), e = the worker's residual of the previous iteration (fp32,
+ *       zero before the first one).
+ *   E2  q_i = 1 if v_i >= 0 (a zero of either sign included), else 0.
+ *   E3  per bucket two reconstruction values, the means of the two classes:
+ *       neg = fl(S0 / c0), pos = fl(S1 / c1) (0 for an empty class; a zero of either sign
+ *       stored as +0).  c = the class's element count; S = its sum in fixed order: rows
+ *       of 32 elements from the bucket's first element, inside a row the chain
+ *       a <- fl(a + v_j) over the row's members of the class from a = 0, left to right,
+ *       and the row sums combined by the balanced tree of adjacent pairs (as N2).
+ *       They are sent as ranges[2k] = neg, ranges[2k + 1] = pos, so that the wire format
+ *       is the (min, max) variant's with K = 1 and the receiver needs nothing new.
+ *   E4  the value the receiver will reconstruct (M4 with K = 1): r = fl(pos - neg);
+ *       x^_i = fma(q_i, r, neg); a bucket with r < 2^-96 is constant: codes 0, x^ = neg.
+ *   E5  e_i <- fl(v_i - x^_i): the residual is taken against E4's value, not against the
+ *       ideal mean, so nothing the receiver loses is forgotten.
+ */
+static float mqo_class_sum_tree(const float *v, uint64_t len, int cls)
+{
+    uint64_t rows = (len + 31) / 32;
+    uint64_t padded = 1;
+    while (padded < rows) padded *= 2;
+    float *node = (float *)calloc(padded, sizeof(float));
+    if (!node) return NAN;
+    for (uint64_t r = 0; r < rows; ++r) {
+        uint64_t j0 = 32 * r, j1 = j0 + 32;
+        if (j1 > len) j1 = len;
+        float a = 0.0f;
+        for (uint64_t j = j0; j < j1; ++j)
+            if ((v[j] >= 0.0f ? 1 : 0) == cls) a = a + v[j];
+        node[r] = a;
+    }
+    for (uint64_t width = padded; width > 1; width /= 2)
+        for (uint64_t j = 0; j < width / 2; ++j)
+            node[j] = node[2 * j] + node[2 * j + 1];
+    float S = node[0];
+    free(node);
+    return S;
+}
+
+/* E1..E5 for one worker buffer; residual is read and overwritten.  dtype as mqo_quantize. */
+int mqo_quantize_1bit_ef(const void *grad, float *residual, uint64_t n, uint64_t bucket,
+                         uint32_t *codes, float *ranges, int dtype)
+{
+    if (bucket == 0) return -1;
+    if (n == 0) return 0;
+    const float tiny = ldexpf(1.0f, -96);
+    float *v = (float *)malloc(n * sizeof(float));
+    uint8_t *q = (uint8_t *)malloc(n);
+    if (!v || !q) { free(v); free(q); return -2; }
+    if (dtype == 1) mqo_widen_bf16((const uint16_t *)grad, n, v);
+    else memcpy(v, grad, n * sizeof(float));
+    for (uint64_t i = 0; i < n; ++i) v[i] = v[i] + residual[i];            /* E1 */
+    uint64_t nb = (n + bucket - 1) / bucket;
+    for (uint64_t k = 0; k < nb; ++k) {
+        uint64_t b0 = k * bucket, b1 = b0 + bucket;
+        if (b1 > n) b1 = n;
+        uint64_t c1 = 0;
+        for (uint64_t i = b0; i < b1; ++i) {                               /* E2 */
+            q[i] = (v[i] >= 0.0f) ? 1 : 0;
+            c1 += q[i];
+        }
+        uint64_t c0 = (b1 - b0) - c1;
+        float S0 = mqo_class_sum_tree(v + b0, b1 - b0, 0);
+        float S1 = mqo_class_sum_tree(v + b0, b1 - b0, 1);
+        float neg = c0 ? S0 / (float)c0 : 0.0f;                            /* E3 */
+        float pos = c1 ? S1 / (float)c1 : 0.0f;
+        neg = neg + 0.0f;
+        pos = pos + 0.0f;
+        ranges[2 * k] = neg;
+        ranges[2 * k + 1] = pos;
+        float r = pos - neg;                                               /* E4 */
+        for (uint64_t i = b0; i < b1; ++i) {
+            if (r < tiny) q[i] = 0;
+            float xhat = (r < tiny) ? neg : fmaf((float)q[i], r, neg);
+            residual[i] = v[i] - xhat;                                     /* E5 */
+        }
+    }
+    mqo_pack(q, n, 1, codes);
+    free(v); free(q);
     return 0;
 }

@@ -335,3 +335,21 @@ def quantize_segments_l2(grad, seg_off, code_off, bits, seed, worker=0, step=0, 
     if rc:
         raise ValueError("mqo_quantize_segments_l2 failed: %d" % rc)
     return codes, scales
+
+
+# ---- codec variant: one bit per element with error feedback ----------------------------------
+_q1ef = _decl("mqo_quantize_1bit_ef", _int, _vp, _vp, _u64, _u64, _vp, _vp, _int)
+
+
+def quantize_1bit_ef(grad, residual, bucket, dtype="f32"):
+    """Returns (codes, ranges, new residual); `residual` itself is not modified."""
+    grad = _c(grad, np.uint16 if dtype == "bf16" else np.float32)
+    n = grad.size
+    res = np.array(residual, np.float32, copy=True)
+    assert res.size == n
+    codes = np.zeros(code_words(n, 1), np.uint32)
+    ranges = np.zeros(2 * num_buckets(n, bucket) if n else 0, np.float32)
+    rc = _q1ef(_ptr(grad), _ptr(res), n, bucket, _ptr(codes), _ptr(ranges), 1 if dtype == "bf16" else 0)
+    if rc:
+        raise ValueError("mqo_quantize_1bit_ef failed: %d" % rc)
+    return codes, ranges, res
