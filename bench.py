@@ -555,6 +555,33 @@ def run_ours(args):
                      "roofline": {"bound": "hbm", "achieved": l2_q_bytes / l2_q_s / 1e9, "peak": peak, "unit": "GB/s",
                                   "frac": l2_q_bytes / l2_q_s / 1e9 / peak, "traffic": None}},
     }
+    # ---- codec variant (outside `value`): one bit with error feedback; the quantizer reads the gradient and
+    # the residual and writes the residual back (12 + 1/8 + 8/B bytes per element); the server step is the
+    # (min, max) variant's with one bit
+    ef_res = [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(W)]
+
+    def ef_quantize():
+        for w in range(W):
+            check(lib.mqg_quantize_1bit_ef(grads[w].data_ptr(), ef_res[w].data_ptr(), n, B,
+                                           codes[1][w].data_ptr(), mm_ranges[w].data_ptr(), 0, sptr))
+
+    ef_quantize()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for i in range(mm_steps):
+        ef_quantize()
+    f1.record(stream)
+    torch.cuda.synchronize()
+    ef_s = f0.elapsed_time(f1) * 1e-3 / mm_steps
+    ef_bytes = W * (12 * n + 4 * mqg.mqg_code_words(n, 1) + 8 * mqg.mqg_num_buckets(n, B))
+    variant_1bit_ef = {
+        "codec": "one bit per element with error feedback (mqg_quantize_1bit_ef; server step = the (min, max) "
+                 "variant's with bits = 1); not part of `value`",
+        "quantize": {"avg_launch_us": ef_s / W * 1e6, "launches_per_step": W,
+                     "roofline": {"bound": "hbm", "achieved": ef_bytes / ef_s / 1e9, "peak": peak, "unit": "GB/s",
+                                  "frac": ef_bytes / ef_s / 1e9 / peak, "traffic": None}},
+    }
+    del ef_res
     # put the codes back as the main codec writes them (the end-to-end leg re-quantizes anyway)
     for b in ALL_BITS:
         quantize_all(b, 0)
@@ -589,6 +616,7 @@ def run_ours(args):
             "gpu_launches": args.steps * len(ALL_BITS) * (q_launches + 1),
             "roofline": roofline, "roofline_server": roofline_server, "downlink": downlink_line,
             "variant_minmax": variant_minmax, "variant_l2": variant_l2,
+            "variant_1bit_ef": variant_1bit_ef,
             "per_bits": per_bits,
         }
         if cpu is not None:

@@ -171,6 +171,29 @@ mqg_status mqg_server_step_minmax(const uint32_t* const* codes, const float* con
                                   void* cuda_stream);
 
 /*
+ * Codec variant: one bit per element with error feedback, the 1-bit scheme that the related-work
+ * section (Section 2) cites: the sign of every value is sent and the quantization error is carried
+ * into the next mini-batch.  With e the worker's residual (n floats kept by the caller from one
+ * iteration to the next, zero before the first):
+ *     v = fl(g + e);   code = 1 if v >= 0 (a zero of either sign included) else 0
+ *     per bucket: neg = mean of v over the elements with code 0, pos = mean over those with code 1
+ *                 (0 for an empty class), written as ranges[2b] = neg, ranges[2b + 1] = pos
+ *     x^ = what mqg_server_step_minmax / mqg_dequant_accumulate_minmax with bits = 1 reconstruct from
+ *          (code, neg, pos): neg for code 0, fl(fl(pos - neg) + neg) for code 1; a bucket with
+ *          fl(pos - neg) < 2^-96 is constant (codes cleared, x^ = neg)
+ *     e <- fl(v - x^)
+ * The class sums are taken in a fixed order (inside a row of 32 elements from the bucket's start a
+ * left-to-right chain over the class's members; the rows' sums by a balanced tree of adjacent
+ * pairs, leaf count padded with zeros to a power of two), so the result is reproducible bit for bit.
+ *   residual [in/out] n floats, 16-byte aligned, updated in place
+ *   codes    [out]    mqg_code_words(n, 1) words;  ranges [out] 2 * mqg_num_buckets(n, bucket) floats,
+ *                     8-byte aligned.  The server side is the (min, max) variant's with bits = 1.
+ * Buckets (or a single bucket n) above 8192 elements are rejected with MQG_ERR_INVALID.
+ */
+mqg_status mqg_quantize_1bit_ef(const void* grad, float* residual, uint64_t n, uint64_t bucket,
+                                uint32_t* codes, float* ranges, mqg_dtype dtype, void* cuda_stream);
+
+/*
  * Codec variant: the bucket's scale is its Euclidean norm, as in the norm-scaled quantizers the
  * related-work section (Section 2) cites, instead of its largest magnitude.  Everything else is
  * mqg_quantize: same encode against [-s, +s], same draws, same packing, and the outputs are

@@ -9,7 +9,7 @@ Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_quantize_minmax,
   mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_segments_l2,
-  mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_code_words, mqg_num_buckets,
+  mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_quantize_1bit_ef, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
 """
 from __future__ import annotations
@@ -61,6 +61,7 @@ def _load() -> C.CDLL:
         "mqg_server_requantize": (i32, [vp, vp, i32, i32, u64, u64, f32, u64, vp, vp, u32, u32, vp]),
         "mqg_quantize_segments": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_server_step_segments": (i32, [vp, vp, i32, i32, i32, vp, vp, vp, f32, vp, vp]),
+        "mqg_quantize_1bit_ef": (i32, [vp, vp, u64, u64, vp, vp, i32, vp]),
         "mqg_quantize_l2": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_l2_workspace_floats": (C.c_size_t, [i32, vp]),
         "mqg_quantize_segments_l2": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp,
@@ -234,6 +235,13 @@ def mqg_server_step_segments(codes, scales, W: int, bits: int, seg_off, code_off
                                          _dev_ptr(params, "params"), lr,
                                          _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
                                          _stream()))
+
+
+def mqg_quantize_1bit_ef(grad, residual, n: int, bucket: int, codes, ranges) -> None:
+    """`residual` (float32, n elements) is read and updated in place."""
+    _check(_lib.mqg_quantize_1bit_ef(_dev_ptr(grad, "grad"), _dev_ptr(residual, "residual"), n, bucket,
+                                     _dev_ptr(codes, "codes"), _dev_ptr(ranges, "ranges"),
+                                     _grad_dtype(grad), _stream()))
 
 
 def mqg_quantize_l2(grad, n: int, bits: int, bucket: int, seed: int, codes, scales,

@@ -390,6 +390,27 @@ mqg_status mqg_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t buck
     return MQG_OK;
 }
 
+mqg_status mqg_quantize_1bit_ef(const void* grad, float* residual, uint64_t n, uint64_t bucket,
+                                uint32_t* codes, float* ranges, mqg_dtype dtype, void* cuda_stream)
+{
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (n == 0) return MQG_OK;
+    if ((bucket < n ? bucket : n) > (uint64_t)mqg::kMaxFusedBucket)
+        return fail(MQG_ERR_INVALID, "mqg_quantize_1bit_ef supports buckets of at most %d elements",
+                    mqg::kMaxFusedBucket);
+    if (!grad || !residual || !codes || !ranges)
+        return fail(MQG_ERR_INVALID, "grad, residual, codes or ranges is null");
+    if (!aligned16(grad)) return fail(MQG_ERR_ALIGN, "grad not 16-byte aligned");
+    if (!aligned16(residual)) return fail(MQG_ERR_ALIGN, "residual not 16-byte aligned");
+    if (!aligned16(codes)) return fail(MQG_ERR_ALIGN, "codes not 16-byte aligned");
+    if (!aligned8(ranges)) return fail(MQG_ERR_ALIGN, "ranges not 8-byte aligned");
+    const cudaError_t err = mqg::launch_quantize_onebit_ef(grad, residual, n, bucket, codes, ranges, (int)dtype,
+                                                           static_cast<cudaStream_t>(cuda_stream));
+    if (err != cudaSuccess) return cuda_fail("mqg_quantize_1bit_ef", err);
+    return MQG_OK;
+}
+
 size_t mqg_l2_workspace_floats(int nseg, const uint64_t* seg_off)
 {
     if (nseg <= 0 || !seg_off) return 0;

@@ -81,6 +81,11 @@ cudaError_t launch_quantize_segments_l2(const void* grad, const SegmentTable& ta
                                         uint32_t step, uint64_t elem_offset, float* partial,
                                         cudaStream_t stream);
 
+// 1-bit error-feedback variant: sign codes, class means as (neg, pos) ranges, residual updated in
+// place.  Buckets of at most kMaxFusedBucket elements.
+cudaError_t launch_quantize_onebit_ef(const void* grad, float* residual, uint64_t n, uint64_t bucket,
+                                      uint32_t* codes, float* ranges, int dtype, cudaStream_t stream);
+
 // Two-pass quantize with uniform large buckets (bucket > kMaxFusedBucket, or a single bucket
 // whose length is not a multiple of 32).
 cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, uint64_t bucket,

@@ -1,5 +1,6 @@
 """Plants single mistakes in a copy of the CPU checker and verifies that the pin
-suites (tests/test_oracle_pins.py, tests/test_oracle_minmax_pins.py, tests/test_oracle_l2_pins.py) reject every one of them.  Everything here runs
+suites (tests/test_oracle_pins.py, tests/test_oracle_minmax_pins.py, tests/test_oracle_l2_pins.py,
+tests/test_oracle_onebit_pins.py) reject every one of them.  Everything here runs
 on the CPU; the planted copies are compiled into a temporary directory."""
 import os
 import subprocess
@@ -81,6 +82,25 @@ MUTANTS_L2 = [
     ("l2_scale_is_max_abs", "mqo_bucket_norms(x, n, bucket, scales);\n    mqo_draw_h", "mqo_bucket_scales(x, n, bucket, scales);\n    mqo_draw_h"),
 ]
 
+# mistakes planted in the 1-bit error-feedback variant, caught by tests/test_oracle_onebit_pins.py
+MUTANTS_ONEBIT = [
+    ("ob_old_residual_ignored", "v[i] = v[i] + residual[i];", "v[i] = v[i];"),
+    ("ob_zero_counts_as_negative", "q[i] = (v[i] >= 0.0f) ? 1 : 0;", "q[i] = (v[i] > 0.0f) ? 1 : 0;"),
+    ("ob_residual_against_ideal_mean", "float xhat = (r < tiny) ? neg : fmaf((float)q[i], r, neg);",
+     "float xhat = (r < tiny) ? neg : (q[i] ? pos : neg);"),
+    ("ob_residual_sign", "residual[i] = v[i] - xhat;", "residual[i] = xhat - v[i];"),
+    ("ob_mean_over_whole_bucket", "float pos = c1 ? S1 / (float)c1 : 0.0f;", "float pos = c1 ? S1 / (float)(b1 - b0) : 0.0f;"),
+    ("ob_ranges_swapped", "ranges[2 * k] = neg;\n        ranges[2 * k + 1] = pos;",
+     "ranges[2 * k] = pos;\n        ranges[2 * k + 1] = neg;"),
+    ("ob_rows_summed_in_sequence",
+     "        node[r] = a;\n    }\n    for (uint64_t width = padded; width > 1; width /= 2)\n"
+     "        for (uint64_t j = 0; j < width / 2; ++j)\n            node[j] = node[2 * j] + node[2 * j + 1];\n    float S = node[0];\n    free(node);\n    return S;\n}\n\n/* E1..E5",
+     "        node[r] = a;\n    }\n    for (uint64_t j = 1; j < padded; ++j) node[0] = node[0] + node[j];\n"
+     "    float S = node[0];\n    free(node);\n    return S;\n}\n\n/* E1..E5"),
+    ("ob_class_sum_takes_every_element", "if ((v[j] >= 0.0f ? 1 : 0) == cls) a = a + v[j];", "a = a + v[j];"),
+    ("ob_constant_bucket_keeps_codes", "if (r < tiny) q[i] = 0;", ""),
+]
+
 
 def _run(args):
     name, old, new, tmpdir = args
@@ -95,7 +115,8 @@ def _run(args):
                     "-shared", "-o", so, c, "-lm"], check=True)
     env = dict(os.environ, MQG_ORACLE_LIB=so)
     pins = ("test_oracle_minmax_pins.py" if name.startswith("mm_")
-            else "test_oracle_l2_pins.py" if name.startswith("l2_") else "test_oracle_pins.py")
+            else "test_oracle_l2_pins.py" if name.startswith("l2_")
+            else "test_oracle_onebit_pins.py" if name.startswith("ob_") else "test_oracle_pins.py")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         os.path.join(ROOT, "tests", pins)],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
@@ -103,7 +124,7 @@ def _run(args):
 
 
 def test_every_planted_mistake_is_caught(tmp_path):
-    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS + MUTANTS_MINMAX + MUTANTS_L2]
+    jobs = [(n, o, w, str(tmp_path)) for n, o, w in MUTANTS + MUTANTS_MINMAX + MUTANTS_L2 + MUTANTS_ONEBIT]
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 2)) as ex:
         results = list(ex.map(_run, jobs))
     survivors = [name for name, rc, _ in results if rc == 0]
