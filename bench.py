@@ -53,7 +53,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per element of quantize_workers_kernel<4> (ncu, 4 x 8,388,608
 # elements): (134.25 MB + 7.82 MB) / 33,554,432; writes are partly still in L2 when the kernel ends
-QUANTIZE_DRAM_BYTES_PER_ELEM_K4 = 142.07e6 / 33_554_432
+QUANTIZE_DRAM_BYTES_PER_ELEM_K4 = 142.48e6 / 33_554_432
 
 
 def measured_hbm_peak():

@@ -59,3 +59,39 @@ def test_full_size_step(bits):
     assert max_rel_err(got, p_ref) <= 1e-6
     assert bits_equal(got, p_ref) == 0
     assert mqg.mqg_device_timeouts() == 0
+
+
+@pytest.mark.parametrize("bits", [1, 5])
+def test_full_size_l2_norm_variant(bits):
+    """The L2-norm scale variant in the launch shape the benchmark times (one launch per worker)."""
+    c = _inputs()
+    workers = (0, 5)
+    with ThreadPoolExecutor(2) as ex:
+        ref = list(ex.map(lambda w: O.quantize_l2(c["host"][w], bits, B, SEED, worker=w, step=7), workers))
+    for (c_ref, s_ref), w in zip(ref, workers):
+        dc = Guarded(mqg.mqg_code_words(N, bits), torch.int32)
+        ds = Guarded(mqg.mqg_num_buckets(N, B), torch.float32)
+        mqg.mqg_quantize_l2(c["dev"][w], N, bits, B, SEED, dc.view, ds.view, worker=w, step=7)
+        torch.cuda.synchronize()
+        dc.check_guards(), ds.check_guards()
+        assert bits_equal(ds.numpy(np.float32), s_ref) == 0
+        assert np.array_equal(dc.numpy(np.uint32), c_ref)
+    assert mqg.mqg_device_timeouts() == 0
+
+
+def test_full_size_one_bit_error_feedback_variant():
+    """Two iterations of the 1-bit error-feedback quantizer on one worker's full-size gradient."""
+    c = _inputs()
+    g, g_dev = c["host"][3], c["dev"][3]
+    res = Guarded(N, torch.float32, fill=np.zeros(N, np.float32))
+    e_ref = np.zeros(N, np.float32)
+    for it in range(2):
+        dc = Guarded(mqg.mqg_code_words(N, 1), torch.int32)
+        dr = Guarded(2 * mqg.mqg_num_buckets(N, B), torch.float32)
+        mqg.mqg_quantize_1bit_ef(g_dev, res.view, N, B, dc.view, dr.view)
+        torch.cuda.synchronize()
+        dc.check_guards(), dr.check_guards(), res.check_guards()
+        c_ref, r_ref, e_ref = O.quantize_1bit_ef(g, e_ref, B)
+        assert bits_equal(dr.numpy(np.float32), r_ref) == 0
+        assert np.array_equal(dc.numpy(np.uint32), c_ref)
+        assert bits_equal(res.numpy(np.float32), e_ref) == 0
