@@ -350,6 +350,10 @@ def run_ours(args):
             p2.record(stream)
             phases.append((p0, p1, p2))
 
+    # The read-back of the updated parameters runs on its own stream, so that it shares the (full-duplex)
+    # host link with the next bit width's gradient upload instead of waiting in front of it.
+    d2h_stream = torch.cuda.Stream()
+
     def e2e_step(step_no):
         for b in ALL_BITS:
             for w in range(W):
@@ -357,7 +361,12 @@ def run_ours(args):
                 check(lib.mqg_quantize(grads[w].data_ptr(), n, b, B, PHILOX_SEED, codes[b][w].data_ptr(),
                                        scales[b][w].data_ptr(), 0, w, step_no, 0, sptr))
             server(b)
-            host_params.copy_(params[b], non_blocking=True)
+            updated = torch.cuda.Event()
+            updated.record(stream)
+            d2h_stream.wait_event(updated)
+            with torch.cuda.stream(d2h_stream):
+                host_params.copy_(params[b], non_blocking=True)
+        stream.wait_stream(d2h_stream)             # the step ends when its last result is on the host
 
     def barrier():
         torch.cuda.synchronize()
@@ -629,7 +638,8 @@ def run_ours(args):
 
 def run_single_kernel(args):
     """A few launches of one kernel on a small case (inputs still larger than L2), for profiler
-    captures and quick timing: python bench.py --kernel quantize|quantize_workers|server --bits B [--n N]."""
+    captures and quick timing: python bench.py --kernel quantize|quantize_workers|server|requantize|quantize_l2|onebit
+    --bits B [--n N]."""
     import torch
 
     import paper_1804_08066_b200 as mqg
@@ -646,6 +656,22 @@ def run_single_kernel(args):
         launch = lambda i: mqg.mqg_quantize(grads[i % rot], n, b, B, PHILOX_SEED, codes[i % rot],
                                             scales[i % rot], worker=i % rot, step=i)
         nbytes = quantize_bytes(n, b, B)
+    elif args.kernel == "quantize_l2":
+        grads = [torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w)).cuda() for w in range(rot)]
+        codes = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
+        scales = [torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize_l2(grads[i % rot], n, b, B, PHILOX_SEED, codes[i % rot],
+                                               scales[i % rot], worker=i % rot, step=i)
+        nbytes = quantize_bytes(n, b, B)
+    elif args.kernel == "onebit":
+        b = 1
+        grads = [torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w)).cuda() for w in range(rot)]
+        resid = [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(rot)]
+        codes = [torch.zeros(mqg.mqg_code_words(n, 1), dtype=torch.int32, device="cuda") for _ in range(rot)]
+        ranges = [torch.zeros(2 * mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize_1bit_ef(grads[i % rot], resid[i % rot], n, B, codes[i % rot],
+                                                    ranges[i % rot])
+        nbytes = 12 * n + 4 * mqg.mqg_code_words(n, 1) + 8 * mqg.mqg_num_buckets(n, B)
     elif args.kernel == "quantize_workers":
         # W gradients of n elements per launch; two buffer sets, each far larger than L2
         rot = 2
@@ -709,7 +735,8 @@ def main():
     ap.add_argument("--quantize-launch", choices=["batched", "per-worker"], default="batched",
                     help="the step's quantize phase: one mqg_quantize_workers launch per bit width for all "
                          "workers' gradients, or one mqg_quantize launch per worker")
-    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize"], default=None,
+    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize", "quantize_l2", "onebit"],
+                    default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--n", type=int, default=1 << 25)
