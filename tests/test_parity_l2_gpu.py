@@ -88,9 +88,11 @@ def test_quantize_bf16(bits):
     assert_quantize_parity(x[:8001], bits, 1 << 20, bf16=True, seed=2)
 
 
-def test_unaligned_element_offset():
+def test_element_offsets():
     x = wl.normal(10_000, 1e-2, config=1, worker=5)
-    assert_quantize_parity(x, 5, 1024, seed=11, worker=1, step=2, elem_offset=12_345)
+    assert_quantize_parity(x, 5, 1024, seed=11, worker=1, step=2, elem_offset=12_345)       # not a multiple of 8
+    assert_quantize_parity(x, 5, 1024, seed=11, worker=1, step=2, elem_offset=8 * 12_345)   # block-aligned
+    assert_quantize_parity(x, 2, 4096, seed=(1 << 40) + 3, worker=7, step=9, elem_offset=(1 << 36) + 64)
 
 
 def test_buckets_above_the_one_pass_limit_are_rejected():
