@@ -557,15 +557,6 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
             for (int p = 0; p < 16; ++p)
                 v2[p] = accumulate2<8, RANGE>(v2[p], make_float2(byte_to_biased(w[p >> 1], (2 * p) & 3, bias),
                                                           byte_to_biased(w[p >> 1], (2 * p + 1) & 3, bias)), th, mh);
-        } else if constexpr (BITS == 4) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const uint32_t lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
-#pragma unroll
-                for (int b = 0; b < 4; ++b)      // elements 8k + 2b (low nibble) and 8k + 2b + 1 (high)
-                    v2[4 * k + b] = accumulate2<4, RANGE>(v2[4 * k + b],
-                                                   make_float2(byte_to_biased(lo, b, bias), byte_to_biased(hi, b, bias)), th, mh);
-            }
         } else if constexpr (BITS == 2) {
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
@@ -581,11 +572,39 @@ __device__ __forceinline__ void add_decoded_row(const uint32_t (&w)[BITS], const
                 }
             }
         } else {
+            // Widths 3 to 7 (and width 1 of the range variant).  A group of G consecutive codes is
+            // brought to bit 0 with one (funnel) shift; code g of the group is then masked IN PLACE
+            // into the mantissa of 2^23, which gives the float 2^23 + q * 2^(g K) (g K + K <= 23), and
+            // one packed fma with compile-time constants turns two of these into q - off exactly:
+            //     fma(2^23 + q 2^s, 2^-s, -(2^(23 - s) + off)) = q - off      (every term is exact).
+            // One shift per group and one logic operation per code instead of a shift and a logic
+            // operation per code.  off = (L - 1) / 2 for the main codec, 0 for the range variant.
+            // Width 4 measured 54.6 us per launch this way against 56.5 us with nibble masks and byte
+            // permutes (n = 25 M, W = 8), width 3 51.9 against 55.0 us; widths 1 and 2 measured slower
+            // (47.7 against 45.0 us, 47.9 against 47.0 us) and keep their own paths.
+            constexpr int G = 4 * BITS <= 23 ? 4 : 2;
+            constexpr uint32_t kMask = (1u << BITS) - 1u;
+            constexpr float kOff = RANGE ? 0.0f : (float)(((1 << BITS) - 2) / 2);
 #pragma unroll
-            for (int p = 0; p < 16; ++p) {
-                const uint32_t q0 = unpack_one<BITS>(w, 2 * p), q1 = unpack_one<BITS>(w, 2 * p + 1);
-                v2[p] = accumulate2<BITS, RANGE>(v2[p], make_float2(__uint_as_float(q0 | bias),
-                                                             __uint_as_float(q1 | bias)), th, mh);
+            for (int grp = 0; grp < 32 / G; ++grp) {
+                const int o = grp * G * BITS, wi = o >> 5, sh = o & 31;
+                uint32_t win;
+                if (sh == 0) win = w[wi];
+                else if (sh + G * BITS <= 32) win = w[wi] >> sh;
+                else win = __funnelshift_r(w[wi], w[wi + 1], sh);
+#pragma unroll
+                for (int h = 0; h < G / 2; ++h) {
+                    constexpr float kTwo23 = 8388608.0f;
+                    const int s0 = 2 * h * BITS, s1 = s0 + BITS;            // bit positions inside the group
+                    const float2 m = make_float2(__uint_as_float((win & (kMask << s0)) | bias),
+                                                 __uint_as_float((win & (kMask << s1)) | bias));
+                    const float2 scale = make_float2(1.0f / (float)(1u << s0), 1.0f / (float)(1u << s1));
+                    const float2 shift = make_float2(-(kTwo23 / (float)(1u << s0) + kOff),
+                                                     -(kTwo23 / (float)(1u << s1) + kOff));
+                    const float2 qi = __ffma2_rn(m, scale, shift);          // (q - off) for both lanes, exact
+                    const int p = grp * (G / 2) + h;
+                    v2[p] = __fadd2_rn(v2[p], __ffma2_rn(qi, th, mh));
+                }
             }
         }
     }
