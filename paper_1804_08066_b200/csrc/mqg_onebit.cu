@@ -9,9 +9,10 @@
 // left-to-right chain over the members of the class, then the balanced tree over the bucket's
 // rows - and the counts are exact, so the results are reproducible bit for bit.
 //
-// One pass: a CTA stages a tile of whole buckets (up to 256 rows) of v in shared memory with
-// coalesced loads of g and e, every thread owns a row, and the new residual leaves through the
-// same tile with coalesced stores.  12 + 1/8 bytes per element of traffic for almost no arithmetic.
+// One pass: a CTA stages a tile of whole buckets (up to 256 rows) of g and of e in shared memory
+// with 16-byte asynchronous copies (the whole tile in flight at once, nothing through registers),
+// every thread owns a row, and the new residual leaves through e's tile with coalesced stores.
+// 12 + 1/8 bytes per element of traffic for almost no arithmetic.
 #include "mqg_internal.h"
 #include "mqg_tree.cuh"
 
@@ -35,51 +36,65 @@ __device__ __forceinline__ float grad_at(const void* grad, uint64_t i)
     else return bf16_lo(__ldcs(static_cast<const uint16_t*>(grad) + i));
 }
 
-// tile <- g + e for `rows` rows starting at element e0 (a multiple of 32, so 16-byte aligned in
-// every buffer); elements at or beyond n are staged as zeros.
+// 16-byte asynchronous copy global -> shared (no register staging; completion by cp_async_wait_all).
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// tile_g <- g (widened), tile_e <- e for `rows` rows starting at element e0 (a multiple of 32, so
+// 16-byte aligned in every buffer); elements at or beyond n are staged as zeros.  Whole 16-byte
+// chunks travel as asynchronous copies, so a CTA has its entire tile in flight at once.
 template <int DTYPE>
-__device__ __forceinline__ void stage_sum(float4* tile, const OneBitArgs& a, uint64_t e0, int rows)
+__device__ __forceinline__ void stage_tiles(float4* tile_g, float4* tile_e, const OneBitArgs& a, uint64_t e0, int rows)
 {
     const uint64_t valid = a.n - e0;
     const int chunks = rows * 8;
     for (int idx = threadIdx.x; idx < chunks; idx += kMaxTileRows) {
         const uint64_t e = 4ull * idx;
-        float g[4], r[4];
+        const int dst = swz(idx >> 3, idx & 7);
         if (e + 4 <= valid) {
+            cp_async16(&tile_e[dst], a.residual + e0 + e);
             if constexpr (DTYPE == 0) {
-                const float4 gv = __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(a.grad) + e0 + e));
-                g[0] = gv.x; g[1] = gv.y; g[2] = gv.z; g[3] = gv.w;
+                cp_async16(&tile_g[dst], static_cast<const float*>(a.grad) + e0 + e);
             } else {
                 const uint2 gv = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(a.grad) + e0 + e));
-                g[0] = bf16_lo(gv.x); g[1] = bf16_hi(gv.x); g[2] = bf16_lo(gv.y); g[3] = bf16_hi(gv.y);
+                tile_g[dst] = make_float4(bf16_lo(gv.x), bf16_hi(gv.x), bf16_lo(gv.y), bf16_hi(gv.y));
             }
-            const float4 rv = __ldcs(reinterpret_cast<const float4*>(a.residual + e0 + e));
-            r[0] = rv.x; r[1] = rv.y; r[2] = rv.z; r[3] = rv.w;
         } else {
+            float g[4], r[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const bool in = e + k < valid;
                 g[k] = in ? grad_at<DTYPE>(a.grad, e0 + e + k) : 0.0f;
                 r[k] = in ? __ldcs(a.residual + e0 + e + k) : 0.0f;
             }
+            tile_g[dst] = make_float4(g[0], g[1], g[2], g[3]);
+            tile_e[dst] = make_float4(r[0], r[1], r[2], r[3]);
         }
-        tile[swz(idx >> 3, idx & 7)] = make_float4(__fadd_rn(g[0], r[0]), __fadd_rn(g[1], r[1]),
-                                                   __fadd_rn(g[2], r[2]), __fadd_rn(g[3], r[3]));
     }
+    cp_async_wait_all();
 }
+
+constexpr size_t kOneBitSmemBytes = 2 * kMaxTileRows * 128 + 3 * kMaxTileRows * sizeof(float) + 1024;
 
 template <int DTYPE>
 __global__ void __launch_bounds__(kMaxTileRows)
 onebit_ef_kernel(const OneBitArgs a)
 {
-    __shared__ __align__(1024) float4 tile[kMaxTileRows * 8];
-    __shared__ float s_part[3][kMaxTileRows];
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = smem_raw + ((1024u - ((uint32_t)__cvta_generic_to_shared(smem_raw) & 1023u)) & 1023u);
+    float4* tile_g = reinterpret_cast<float4*>(base);
+    float4* tile = tile_g + kMaxTileRows * 8;            // the residual's tile, rewritten in place
+    float (*s_part)[kMaxTileRows] = reinterpret_cast<float (*)[kMaxTileRows]>(tile + kMaxTileRows * 8);
 
     const uint32_t t = threadIdx.x;
     const uint64_t row0 = (uint64_t)blockIdx.x * a.tile_rows;
     const uint64_t rows_left = a.nrows - row0;
     const int rows = (int)(rows_left < a.tile_rows ? rows_left : a.tile_rows);
-    stage_sum<DTYPE>(tile, a, row0 * 32, rows);
+    stage_tiles<DTYPE>(tile_g, tile, a, row0 * 32, rows);
     __syncthreads();
 
     const bool active = t < (uint32_t)rows;
@@ -87,7 +102,11 @@ onebit_ef_kernel(const OneBitArgs a)
     float v[32];
     uint32_t mask = 0u;                          // the row's elements that exist
     if (active) {
+        float g[32];
+        read_row(tile_g, (int)t, g);
         read_row(tile, (int)t, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __fadd_rn(g[j], v[j]);      // v = g + e, one rounding
         const uint64_t left = a.n - row * 32;
         mask = left >= 32 ? 0xFFFFFFFFu : ((1u << (uint32_t)left) - 1u);
     } else {
@@ -153,8 +172,21 @@ cudaError_t launch_quantize_onebit_ef(const void* grad, float* residual, uint64_
     a.tile_rows = a.buckets_per_tile * a.rows_per_bucket;
     const uint64_t ntiles = (a.nrows + a.tile_rows - 1) / a.tile_rows;
     if (ntiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-    if (dtype == 0) onebit_ef_kernel<0><<<(unsigned)ntiles, kMaxTileRows, 0, stream>>>(a);
-    else onebit_ef_kernel<1><<<(unsigned)ntiles, kMaxTileRows, 0, stream>>>(a);
+    static bool configured[2][64] = {};                 // per dtype and device
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dtype != 0][dev]) {
+        err = dtype == 0 ? cudaFuncSetAttribute(onebit_ef_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)kOneBitSmemBytes)
+                         : cudaFuncSetAttribute(onebit_ef_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)kOneBitSmemBytes);
+        if (err != cudaSuccess) return err;
+        configured[dtype != 0][dev] = true;
+    }
+    if (dtype == 0) onebit_ef_kernel<0><<<(unsigned)ntiles, kMaxTileRows, kOneBitSmemBytes, stream>>>(a);
+    else onebit_ef_kernel<1><<<(unsigned)ntiles, kMaxTileRows, kOneBitSmemBytes, stream>>>(a);
     return cudaGetLastError();
 }
 
