@@ -656,6 +656,18 @@ def run_single_kernel(args):
         launch = lambda i: mqg.mqg_quantize(grads[i % rot], n, b, B, PHILOX_SEED, codes[i % rot],
                                             scales[i % rot], worker=i % rot, step=i)
         nbytes = quantize_bytes(n, b, B)
+    elif args.kernel == "quantize_segments":
+        # the layered AlexNet-shaped gradient (16 tensors, one scale per tensor): two passes over the gradient
+        sizes = [int(np.prod(sh)) for sh in wl.ALEXNET_SHAPES]
+        n = sum(sizes)
+        seg = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+        coff = np.concatenate([[0], np.cumsum([mqg.mqg_code_words(sz, b) for sz in sizes])]).astype(np.uint64)
+        grads = [torch.from_numpy(wl.layered(sizes, config=3, worker=w)).cuda() for w in range(rot)]
+        codes = [torch.zeros(int(coff[-1]), dtype=torch.int32, device="cuda") for _ in range(rot)]
+        scales = [torch.zeros(len(sizes), dtype=torch.float32, device="cuda") for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize_segments(grads[i % rot], seg, coff, b, PHILOX_SEED, codes[i % rot],
+                                                     scales[i % rot], worker=i % rot, step=i)
+        nbytes = 8 * n + 4 * int(coff[-1])
     elif args.kernel == "quantize_l2":
         grads = [torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w)).cuda() for w in range(rot)]
         codes = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
@@ -735,7 +747,8 @@ def main():
     ap.add_argument("--quantize-launch", choices=["batched", "per-worker"], default="batched",
                     help="the step's quantize phase: one mqg_quantize_workers launch per bit width for all "
                          "workers' gradients, or one mqg_quantize launch per worker")
-    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize", "quantize_l2", "onebit"],
+    ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize", "quantize_l2", "onebit",
+                             "quantize_segments"],
                     default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)

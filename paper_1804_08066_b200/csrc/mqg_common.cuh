@@ -367,11 +367,22 @@ __device__ __forceinline__ void write_row(float4* tile, int row, const float (&x
         tile[swz(row, c)] = make_float4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
 }
 
+// 16-byte asynchronous copy global -> shared: no register staging, so a thread can have all its
+// chunks of a tile in flight at once; cp_async_wait_all() (then a barrier) before the data is read.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // Cooperative, coalesced copy of a tile of `rows` rows into / out of a swizzled tile.  `src`
 // points at the tile's first element and `valid` is the number of elements that exist from
 // there on (elements at or beyond it read as zero and are never written).  128-bit accesses
 // when the tile's first element is 16-byte aligned, 32-bit (16-bit for bf16) otherwise.
-template <int THREADS>
+// The aligned fp32 path copies asynchronously; with WAIT = false the caller overlaps other work
+// with the copies and calls cp_async_wait_all() itself before the barrier that precedes the reads.
+template <int THREADS, bool WAIT = true>
 __device__ __forceinline__ void load_tile_f32(float4* tile, const float* __restrict__ src,
                                               uint64_t valid, int rows)
 {
@@ -379,16 +390,18 @@ __device__ __forceinline__ void load_tile_f32(float4* tile, const float* __restr
         const int chunks = rows * 8;
         for (int idx = threadIdx.x; idx < chunks; idx += THREADS) {
             const uint64_t e = 4ull * idx;
-            float4 v;
-            if (e + 4 <= valid) v = __ldcs(reinterpret_cast<const float4*>(src + e));
+            float4* dst = &tile[swz(idx >> 3, idx & 7)];
+            if (e + 4 <= valid) cp_async16(dst, src + e);
             else {
+                float4 v;
                 v.x = (e + 0 < valid) ? src[e + 0] : 0.0f;
                 v.y = (e + 1 < valid) ? src[e + 1] : 0.0f;
                 v.z = (e + 2 < valid) ? src[e + 2] : 0.0f;
                 v.w = 0.0f;
+                *dst = v;
             }
-            tile[swz(idx >> 3, idx & 7)] = v;
         }
+        if (WAIT) cp_async_wait_all();
     } else {
         float* tf = reinterpret_cast<float*>(tile);
         const int elems = rows * 32;

@@ -36,14 +36,6 @@ __device__ __forceinline__ float grad_at(const void* grad, uint64_t i)
     else return bf16_lo(__ldcs(static_cast<const uint16_t*>(grad) + i));
 }
 
-// 16-byte asynchronous copy global -> shared (no register staging; completion by cp_async_wait_all).
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
-                 ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
 // tile_g <- g (widened), tile_e <- e for `rows` rows starting at element e0 (a multiple of 32, so
 // 16-byte aligned in every buffer); elements at or beyond n are staged as zeros.  Whole 16-byte
 // chunks travel as asynchronous copies, so a CTA has its entire tile in flight at once.

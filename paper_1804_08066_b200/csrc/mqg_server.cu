@@ -94,8 +94,9 @@ server_kernel(const ServerArgs a, const SegmentTable tab)
         store_tile_f32<kMaxTileRows>(tile, acc, valid, rows);
     } else {
         float* params = a.params + elem0;
-        load_tile_f32<kMaxTileRows>(tile, params, valid, rows);
+        load_tile_f32<kMaxTileRows, false>(tile, params, valid, rows);    // in flight during the decode
         if (active) accumulate_row<BITS, !SEG>(a, scale_idx, word0, words_end, full_row, v, false);
+        cp_async_wait_all();
         __syncthreads();
         if (active) {
             float p[32];
