@@ -668,6 +668,22 @@ def run_single_kernel(args):
         launch = lambda i: mqg.mqg_quantize_segments(grads[i % rot], seg, coff, b, PHILOX_SEED, codes[i % rot],
                                                      scales[i % rot], worker=i % rot, step=i)
         nbytes = 8 * n + 4 * int(coff[-1])
+    elif args.kernel == "server_segments":
+        # fused server step on the layered gradient (per-layer scale), W workers
+        sizes = [int(np.prod(sh)) for sh in wl.ALEXNET_SHAPES]
+        n = sum(sizes)
+        seg = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+        coff = np.concatenate([[0], np.cumsum([mqg.mqg_code_words(sz, b) for sz in sizes])]).astype(np.uint64)
+        g = torch.from_numpy(wl.layered(sizes, config=3, worker=0)).cuda()
+        codes = [[torch.zeros(int(coff[-1]), dtype=torch.int32, device="cuda") for _ in range(W)] for _ in range(rot)]
+        scales = [[torch.zeros(len(sizes), dtype=torch.float32, device="cuda") for _ in range(W)] for _ in range(rot)]
+        for r in range(rot):
+            for w in range(W):
+                mqg.mqg_quantize_segments(g, seg, coff, b, PHILOX_SEED, codes[r][w], scales[r][w], worker=w, step=r)
+        params = [torch.from_numpy(wl.params(n, 0.05, config=3)).cuda() for _ in range(rot)]
+        launch = lambda i: mqg.mqg_server_step_segments(codes[i % rot], scales[i % rot], W, b, seg, coff,
+                                                        params[i % rot], LR)
+        nbytes = 8 * n + W * 4 * int(coff[-1])
     elif args.kernel == "quantize_l2":
         grads = [torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w)).cuda() for w in range(rot)]
         codes = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
@@ -748,7 +764,7 @@ def main():
                     help="the step's quantize phase: one mqg_quantize_workers launch per bit width for all "
                          "workers' gradients, or one mqg_quantize launch per worker")
     ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize", "quantize_l2", "onebit",
-                             "quantize_segments"],
+                             "quantize_segments", "server_segments"],
                     default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)

@@ -2,6 +2,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "../../include/mqgrad.h"
 #include "mqg_common.cuh"
@@ -66,10 +67,11 @@ mqg_status check_workers(const uint32_t* const* codes, const float* const* scale
 }
 
 // Validates a segment table and cuts it into chunks of at most kMaxSegmentsPerLaunch segments;
-// calls fn(table, first_segment_index) for each chunk that has at least one tile.
+// calls fn(table, first_segment_index) for each chunk.  Segments with skip[j] != 0 (skip may be
+// null) get no tiles in the tables, exactly like empty segments: another launch takes care of them.
 template <typename Fn>
 mqg_status for_each_chunk(int nseg, const uint64_t* seg_off, const uint64_t* code_off, int bits,
-                          Fn&& fn)
+                          Fn&& fn, const char* skip = nullptr)
 {
     if (nseg < 0) return fail(MQG_ERR_INVALID, "nseg = %d is negative", nseg);
     if (nseg == 0) return MQG_OK;
@@ -91,7 +93,7 @@ mqg_status for_each_chunk(int nseg, const uint64_t* seg_off, const uint64_t* cod
         uint64_t tiles = 0;
         while (j + k < nseg && k < mqg::kMaxSegmentsPerLaunch) {
             const uint64_t len = seg_off[j + k + 1] - seg_off[j + k];
-            const uint64_t t = (len + tile_elems - 1) / tile_elems;
+            const uint64_t t = (skip && skip[j + k]) ? 0 : (len + tile_elems - 1) / tile_elems;
             if (tiles + t > 0x7FFFFFFFull) break;
             tab.tile_start[k] = (uint32_t)tiles;
             tab.seg_off[k] = seg_off[j + k];
@@ -470,13 +472,43 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
         if (acc_out && !aligned16(acc_out)) return fail(MQG_ERR_ALIGN, "acc_out not 16-byte aligned");
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    return for_each_chunk(nseg, seg_off, code_off, bits,
+    // A long segment is a gradient with a single bucket: it goes to the TMA-fed server kernel in a
+    // launch of its own when its buffers are aligned for bulk copies; all other segments share the
+    // table-driven launch.  The results are the same bit for bit either way.
+    constexpr uint64_t kOwnLaunchElems = 1ull << 20;
+    std::vector<char> own;
+    if (nseg > 0 && seg_off && code_off && !acc_out) {
+        own.assign((size_t)nseg, 0);
+        for (int j = 0; j < nseg; ++j) {
+            if (seg_off[j + 1] < seg_off[j]) break;            // reported by the table check below
+            const uint64_t len = seg_off[j + 1] - seg_off[j];
+            if (len < kOwnLaunchElems || !mqg::server_tma_applies(len, len)) continue;
+            bool aligned = aligned16(params + seg_off[j]);
+            for (int w = 0; w < W && aligned; ++w) aligned = aligned16(codes[w] + code_off[j]);
+            own[(size_t)j] = aligned ? 1 : 0;
+        }
+    }
+    const mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
         [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
             const cudaError_t err = mqg::launch_server_segments(ptrs, W, bits, tab, first, params,
                                                                 lr, acc_out, stream);
             if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
             return MQG_OK;
-        });
+        }, own.empty() ? nullptr : own.data());
+    if (st != MQG_OK) return st;
+    for (int j = 0; j < nseg && !own.empty(); ++j) {
+        if (!own[(size_t)j]) continue;
+        mqg::WorkerPtrs seg_ptrs = ptrs;
+        for (int w = 0; w < W; ++w) {
+            seg_ptrs.codes[w] = codes[w] + code_off[j];
+            seg_ptrs.scales[w] = scales[w] + j;
+        }
+        const uint64_t len = seg_off[j + 1] - seg_off[j];
+        const cudaError_t err = mqg::launch_server(seg_ptrs, W, bits, len, len, params + seg_off[j], lr,
+                                                   nullptr, 0, stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
+    }
+    return MQG_OK;
 }
 
 }  // extern "C"

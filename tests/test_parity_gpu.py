@@ -279,6 +279,29 @@ def test_segments_quantize_and_server(bits):
     assert bits_equal(acc.numpy(np.float32), acc_ref) == 0
 
 
+@pytest.mark.parametrize("bits", [1, 3, 8])
+def test_segments_server_long_segments_take_their_own_launch(bits):
+    """Segments of a million elements and more go to the TMA-fed kernel when their buffers are
+    16-byte aligned (the second one here, ragged length included) and stay in the table-driven
+    launch otherwise (the fourth one starts on an odd word); both must match the checker."""
+    sizes = [128, (1 << 20) + 37, 5, (1 << 20) + 64, 100]
+    W = 3
+    seg, coff = _segments(sizes, bits)
+    n = int(seg[-1])
+    xs = [wl.layered(sizes, config=3, worker=w) for w in range(W)]
+    refs = [O.quantize_segments(x, seg, coff, bits, seed=5, worker=w) for w, x in enumerate(xs)]
+    codes, scales = [r[0] for r in refs], [r[1] for r in refs]
+    p0 = wl.params(n, 0.05, config=3)
+    p_ref, _ = O.server_step_segments(codes, scales, bits, seg, coff, p0.copy(), 0.05)
+    p = Guarded(n, torch.float32, fill=p0)
+    mqg.mqg_server_step_segments([to_dev(c.view(np.int32)) for c in codes], [to_dev(s) for s in scales],
+                                 W, bits, seg, coff, p.view, 0.05)
+    torch.cuda.synchronize()
+    p.check_guards()
+    assert bits_equal(p.numpy(np.float32), p_ref) == 0
+    assert mqg.mqg_device_timeouts() == 0
+
+
 def test_segments_more_than_one_launch_chunk():
     rng = np.random.default_rng(0)
     sizes = [int(v) for v in rng.integers(0, 600, 150)]
