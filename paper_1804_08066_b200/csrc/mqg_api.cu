@@ -2,7 +2,6 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
-#include <vector>
 
 #include "../../include/mqgrad.h"
 #include "mqg_common.cuh"
@@ -67,11 +66,14 @@ mqg_status check_workers(const uint32_t* const* codes, const float* const* scale
 }
 
 // Validates a segment table and cuts it into chunks of at most kMaxSegmentsPerLaunch segments;
-// calls fn(table, first_segment_index) for each chunk.  Segments with skip[j] != 0 (skip may be
-// null) get no tiles in the tables, exactly like empty segments: another launch takes care of them.
-template <typename Fn>
+// calls fn(table, first_segment_index) for each chunk.  Segments for which skip(j) holds get no
+// tiles in the tables, exactly like empty segments: another launch takes care of them.  skip is
+// only called once the table has been checked.
+struct SkipNone { bool operator()(int) const { return false; } };
+
+template <typename Fn, typename Skip = SkipNone>
 mqg_status for_each_chunk(int nseg, const uint64_t* seg_off, const uint64_t* code_off, int bits,
-                          Fn&& fn, const char* skip = nullptr)
+                          Fn&& fn, Skip&& skip = Skip())
 {
     if (nseg < 0) return fail(MQG_ERR_INVALID, "nseg = %d is negative", nseg);
     if (nseg == 0) return MQG_OK;
@@ -93,7 +95,7 @@ mqg_status for_each_chunk(int nseg, const uint64_t* seg_off, const uint64_t* cod
         uint64_t tiles = 0;
         while (j + k < nseg && k < mqg::kMaxSegmentsPerLaunch) {
             const uint64_t len = seg_off[j + k + 1] - seg_off[j + k];
-            const uint64_t t = (skip && skip[j + k]) ? 0 : (len + tile_elems - 1) / tile_elems;
+            const uint64_t t = skip(j + k) ? 0 : (len + tile_elems - 1) / tile_elems;
             if (tiles + t > 0x7FFFFFFFull) break;
             tab.tile_start[k] = (uint32_t)tiles;
             tab.seg_off[k] = seg_off[j + k];
@@ -360,14 +362,38 @@ mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg
         if (!aligned4(scales)) return fail(MQG_ERR_ALIGN, "scales not 4-byte aligned");
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    return for_each_chunk(nseg, seg_off, code_off, bits,
+    // Max pass over every segment; then the encode pass.  A long segment whose buffers are aligned
+    // for bulk copies is encoded by the TMA-fed quantize kernel in a launch of its own (its scale is
+    // final by then); in the table-driven encode launch it has no tiles.  Same results bit for bit.
+    const size_t esz = dtype == MQG_BF16 ? 2 : 4;
+    auto own = [&](int j) {
+        return mqg::quantize_given_scale_applies(static_cast<const char*>(grad) + seg_off[j] * esz,
+                                                 seg_off[j + 1] - seg_off[j], codes + code_off[j],
+                                                 elem_offset + seg_off[j]);
+    };
+    mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
         [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
-            const cudaError_t err = mqg::launch_quantize_segments(grad, tab, bits, seed, codes,
-                                                                  scales + first, (int)dtype, worker,
-                                                                  step, elem_offset, stream);
+            const cudaError_t err = mqg::launch_segments_absmax(grad, tab, scales + first, (int)dtype, stream);
             if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments", err);
             return MQG_OK;
         });
+    if (st != MQG_OK) return st;
+    st = for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            const cudaError_t err = mqg::launch_segments_encode(grad, tab, bits, seed, codes, scales + first,
+                                                                (int)dtype, worker, step, elem_offset, stream);
+            if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments", err);
+            return MQG_OK;
+        }, own);
+    if (st != MQG_OK) return st;
+    for (int j = 0; j < nseg; ++j) {
+        if (!own(j)) continue;
+        const cudaError_t err = mqg::launch_quantize_given_scale(
+            static_cast<const char*>(grad) + seg_off[j] * esz, seg_off[j + 1] - seg_off[j], bits, seed,
+            codes + code_off[j], scales + j, (int)dtype, worker, step, elem_offset + seg_off[j], stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments", err);
+    }
+    return MQG_OK;
 }
 
 mqg_status mqg_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
@@ -445,17 +471,40 @@ mqg_status mqg_quantize_segments_l2(const void* grad, int nseg, const uint64_t* 
         if (!aligned4(workspace)) return fail(MQG_ERR_ALIGN, "workspace not 4-byte aligned");
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // Sums and scales of every segment first; then the encode, where a long segment with buffers
+    // aligned for bulk copies takes a launch of the TMA-fed quantize kernel of its own.
+    const size_t esz = dtype == MQG_BF16 ? 2 : 4;
+    auto own = [&](int j) {
+        return mqg::quantize_given_scale_applies(static_cast<const char*>(grad) + seg_off[j] * esz,
+                                                 seg_off[j + 1] - seg_off[j], codes + code_off[j],
+                                                 elem_offset + seg_off[j]);
+    };
     size_t used = 0;                      // tiles of the chunks already launched
-    return for_each_chunk(nseg, seg_off, code_off, bits,
+    mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
         [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
-            const cudaError_t err = mqg::launch_quantize_segments_l2(grad, tab, bits, seed, codes,
-                                                                     scales + first, (int)dtype, worker,
-                                                                     step, elem_offset, workspace + used,
-                                                                     stream);
+            const cudaError_t err = mqg::launch_segments_l2_scales(grad, tab, scales + first, (int)dtype,
+                                                                   workspace + used, stream);
             if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_l2", err);
             used += tab.tile_start[tab.nseg];
             return MQG_OK;
         });
+    if (st != MQG_OK) return st;
+    st = for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            const cudaError_t err = mqg::launch_segments_encode(grad, tab, bits, seed, codes, scales + first,
+                                                                (int)dtype, worker, step, elem_offset, stream);
+            if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_l2", err);
+            return MQG_OK;
+        }, own);
+    if (st != MQG_OK) return st;
+    for (int j = 0; j < nseg; ++j) {
+        if (!own(j)) continue;
+        const cudaError_t err = mqg::launch_quantize_given_scale(
+            static_cast<const char*>(grad) + seg_off[j] * esz, seg_off[j + 1] - seg_off[j], bits, seed,
+            codes + code_off[j], scales + j, (int)dtype, worker, step, elem_offset + seg_off[j], stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_l2", err);
+    }
+    return MQG_OK;
 }
 
 mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* const* scales, int W,
@@ -476,28 +525,23 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
     // launch of its own when its buffers are aligned for bulk copies; all other segments share the
     // table-driven launch.  The results are the same bit for bit either way.
     constexpr uint64_t kOwnLaunchElems = 1ull << 20;
-    std::vector<char> own;
-    if (nseg > 0 && seg_off && code_off && !acc_out) {
-        own.assign((size_t)nseg, 0);
-        for (int j = 0; j < nseg; ++j) {
-            if (seg_off[j + 1] < seg_off[j]) break;            // reported by the table check below
-            const uint64_t len = seg_off[j + 1] - seg_off[j];
-            if (len < kOwnLaunchElems || !mqg::server_tma_applies(len, len)) continue;
-            bool aligned = aligned16(params + seg_off[j]);
-            for (int w = 0; w < W && aligned; ++w) aligned = aligned16(codes[w] + code_off[j]);
-            own[(size_t)j] = aligned ? 1 : 0;
-        }
-    }
+    auto own = [&](int j) {
+        const uint64_t len = seg_off[j + 1] - seg_off[j];
+        if (acc_out || len < kOwnLaunchElems || !mqg::server_tma_applies(len, len)) return false;
+        bool aligned = aligned16(params + seg_off[j]);
+        for (int w = 0; w < W && aligned; ++w) aligned = aligned16(codes[w] + code_off[j]);
+        return aligned;
+    };
     const mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
         [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
             const cudaError_t err = mqg::launch_server_segments(ptrs, W, bits, tab, first, params,
                                                                 lr, acc_out, stream);
             if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
             return MQG_OK;
-        }, own.empty() ? nullptr : own.data());
+        }, own);
     if (st != MQG_OK) return st;
-    for (int j = 0; j < nseg && !own.empty(); ++j) {
-        if (!own[(size_t)j]) continue;
+    for (int j = 0; j < nseg; ++j) {
+        if (!own(j)) continue;
         mqg::WorkerPtrs seg_ptrs = ptrs;
         for (int w = 0; w < W; ++w) {
             seg_ptrs.codes[w] = codes[w] + code_off[j];

@@ -60,15 +60,9 @@ cudaError_t launch_server_range(const WorkerPtrs& ptrs, int W, int bits, uint64_
 cudaError_t launch_server_range_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                                     float* dst, float lr, int mode, cudaStream_t stream);
 
-// Two-pass quantize of segments.  scales_base points at the scale of the table's first segment.
-cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, int bits,
-                                     uint64_t seed, uint32_t* codes, float* scales_base, int dtype,
-                                     uint32_t worker, uint32_t step, uint64_t elem_offset,
-                                     cudaStream_t stream);
-
 // L2-norm scale variant.  Buckets of at most kMaxFusedBucket elements: one pass.  Segments: tile
-// sums into `partial` (one float per tile of the table, in tile order), a fold per segment, then
-// the ordinary encode pass.
+// sums into `partial` (one float per tile of the table, in tile order) and a fold per segment give
+// the scales (launch_segments_l2_scales); the encode is the ordinary segment encode.
 bool quantize_norm_fused_applies(uint64_t n, uint64_t bucket, uint64_t elem_offset);
 cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
                                        uint32_t* codes, float* scales, int dtype, uint32_t worker,
@@ -76,15 +70,26 @@ cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, u
 cudaError_t launch_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
                                uint32_t* codes, float* scales, int dtype, uint32_t worker, uint32_t step,
                                uint64_t elem_offset, cudaStream_t stream);
-cudaError_t launch_quantize_segments_l2(const void* grad, const SegmentTable& tab, int bits, uint64_t seed,
-                                        uint32_t* codes, float* scales_base, int dtype, uint32_t worker,
-                                        uint32_t step, uint64_t elem_offset, float* partial,
-                                        cudaStream_t stream);
+cudaError_t launch_segments_l2_scales(const void* grad, const SegmentTable& tab, float* scales_base, int dtype,
+                                      float* partial, cudaStream_t stream);
 
 // 1-bit error-feedback variant: sign codes, class means as (neg, pos) ranges, residual updated in
 // place.  Buckets of at most kMaxFusedBucket elements.
 cudaError_t launch_quantize_onebit_ef(const void* grad, float* residual, uint64_t n, uint64_t bucket,
                                       uint32_t* codes, float* ranges, int dtype, cudaStream_t stream);
+
+// The two passes of the per-layer quantizer (scales_base points at the scale of the table's first
+// segment), and the encode of ONE long segment (= one
+// bucket whose scale already stands at *scale) on the TMA-fed quantize kernel.
+cudaError_t launch_segments_absmax(const void* grad, const SegmentTable& tab, float* scales_base, int dtype,
+                                   cudaStream_t stream);
+cudaError_t launch_segments_encode(const void* grad, const SegmentTable& tab, int bits, uint64_t seed,
+                                   uint32_t* codes, float* scales_base, int dtype, uint32_t worker,
+                                   uint32_t step, uint64_t elem_offset, cudaStream_t stream);
+bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset);
+cudaError_t launch_quantize_given_scale(const void* grad, uint64_t n, int bits, uint64_t seed, uint32_t* codes,
+                                        float* scale, int dtype, uint32_t worker, uint32_t step,
+                                        uint64_t elem_offset, cudaStream_t stream);
 
 // Two-pass quantize with uniform large buckets (bucket > kMaxFusedBucket, or a single bucket
 // whose length is not a multiple of 32).

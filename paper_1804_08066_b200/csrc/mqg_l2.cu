@@ -141,23 +141,20 @@ cudaError_t launch_l2_bits(const L2Args& a, int dtype, unsigned grid, cudaStream
     return cudaGetLastError();
 }
 
-// partials -> scales -> encode for one table; `partial` has room for ntiles floats.
-cudaError_t three_pass(const SegQuantArgs& a, const SegmentTable& tab, uint64_t ntiles, uint64_t nscales,
-                       int bits, int dtype, float* partial, cudaStream_t stream)
+// partials -> scales for one table; `partial` has room for the table's tiles.
+cudaError_t sums_and_scales(const void* grad, const SegmentTable& tab, float* scales, int dtype, float* partial,
+                            cudaStream_t stream)
 {
-    if (nscales == 0) return cudaSuccess;
-    if (ntiles > 0x7FFFFFFFull || nscales > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-    const unsigned grid = (unsigned)ntiles;
+    const uint32_t ntiles = tab.tile_start[tab.nseg];
+    if (tab.nseg == 0) return cudaSuccess;
     if (ntiles != 0) {
-        if (dtype == 0) l2_partials_kernel<0><<<grid, kMaxTileRows, 0, stream>>>(a.grad, tab, partial);
-        else l2_partials_kernel<1><<<grid, kMaxTileRows, 0, stream>>>(a.grad, tab, partial);
+        if (dtype == 0) l2_partials_kernel<0><<<ntiles, kMaxTileRows, 0, stream>>>(grad, tab, partial);
+        else l2_partials_kernel<1><<<ntiles, kMaxTileRows, 0, stream>>>(grad, tab, partial);
         const cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }
-    l2_finish_kernel<<<(unsigned)nscales, 256, 0, stream>>>(tab, partial, a.scales);
-    const cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess || ntiles == 0) return err;
-    return launch_encode_segments(a, tab, bits, dtype, grid, stream);
+    l2_finish_kernel<<<(unsigned)tab.nseg, 256, 0, stream>>>(tab, partial, scales);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -199,16 +196,10 @@ cudaError_t launch_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t 
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_quantize_segments_l2(const void* grad, const SegmentTable& tab, int bits, uint64_t seed,
-                                        uint32_t* codes, float* scales_base, int dtype, uint32_t worker,
-                                        uint32_t step, uint64_t elem_offset, float* partial,
-                                        cudaStream_t stream)
+cudaError_t launch_segments_l2_scales(const void* grad, const SegmentTable& tab, float* scales_base, int dtype,
+                                      float* partial, cudaStream_t stream)
 {
-    SegQuantArgs a;
-    a.grad = grad; a.codes = codes; a.scales = scales_base; a.elem_offset = elem_offset;
-    a.key.seed_lo = (uint32_t)seed; a.key.seed_hi = (uint32_t)(seed >> 32);
-    a.key.worker = worker; a.key.step = step;
-    return three_pass(a, tab, tab.tile_start[tab.nseg], (uint64_t)tab.nseg, bits, dtype, partial, stream);
+    return sums_and_scales(grad, tab, scales_base, dtype, partial, stream);
 }
 
 }  // namespace mqg

@@ -201,7 +201,11 @@ struct WorkerView {
 // (lane shuffles); otherwise a whole number of warps (one shared-memory atomic per warp).  After
 // the tile's rows are in registers thread 0 calls `refill(stage, bar)` to start the copy that
 // uses the stage next.  Returns false if the tile's copy never landed.
-template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, bool NORM = false, typename Refill>
+// GIVEN: the scale is not computed here: every tile belongs to one bucket whose scale already stands
+// at wv.scales[0] (per-layer quantization after its max or norm pass); no reduction, no scale written
+// except that a raw maximum below the flush limit is replaced by 0 by the first tile.
+template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, bool NORM = false, bool GIVEN = false,
+          typename Refill>
 __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
                                               const QuantizeArgs& a, const TmaQuantizeConsts& c,
                                               uint32_t k, uint32_t tile, Refill&& refill,
@@ -229,7 +233,9 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     }
     uint32_t m;
     uint32_t* slot = sh.slots[k % 3];
-    if constexpr (NORM) {
+    if constexpr (GIVEN) {
+        m = 0u;
+    } else if constexpr (NORM) {
         // L2-norm scale: the fixed tree over the rows' sums of squares - partner distance 1, 2, 4, ...
         // inside the warp, then (buckets of whole warps) the warp sums, one slot per warp
         float ss = row_sum_squares(x);
@@ -249,7 +255,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     }
     if (__syncthreads_or(!ok)) return false;
     if (t == 0) refill(smem_u32(stage), bar);                    // every thread has read the stage
-    if (!SHUFFLE) {
+    if (!SHUFFLE && !GIVEN) {
         if constexpr (NORM) {
             // tree over the bucket's warp sums, zero leaves up to four (plain stores: nothing to reset;
             // the slot array is written again two barriers from here)
@@ -268,10 +274,18 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     if (!active) return true;
 
     float sc = __uint_as_float(m);
-    if constexpr (NORM) sc = sc < flush_limit() ? 0.0f : __fsqrt_rn(sc);     // flush decided on the sum
-    else if (sc < flush_limit()) sc = 0.0f;
-    const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
-    if (scale_writer && (FULL || bucket < a.nbuckets)) wv.scales[bucket] = sc;
+    if constexpr (GIVEN) {
+        sc = __ldg(wv.scales);
+        if (sc < flush_limit()) {        // readers treat the raw and the flushed value alike
+            if (sc != 0.0f && tile == 0 && t == 0) wv.scales[0] = 0.0f;
+            sc = 0.0f;
+        }
+    } else {
+        if constexpr (NORM) sc = sc < flush_limit() ? 0.0f : __fsqrt_rn(sc);     // flush decided on the sum
+        else if (sc < flush_limit()) sc = 0.0f;
+        const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
+        if (scale_writer && (FULL || bucket < a.nbuckets)) wv.scales[bucket] = sc;
+    }
 
     const EncodeScale es = encode_scale<BITS>(sc);
     uint32_t h[16];
@@ -375,8 +389,9 @@ __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THR
     return true;
 }
 
-// MODE: kMaxAbs = the main codec, kRange = the (min, max) variant, kNorm = the L2-norm scale variant.
-enum : int { kMaxAbs = 0, kRange = 1, kNorm = 2 };
+// MODE: kMaxAbs = the main codec, kRange = the (min, max) variant, kNorm = the L2-norm scale variant,
+// kGiven = encode against a scale computed by an earlier pass (long segments of the per-layer quantizers).
+enum : int { kMaxAbs = 0, kRange = 1, kNorm = 2, kGiven = 3 };
 
 template <int BITS, int DTYPE, int THREADS, bool SHUFFLE, int MODE = kMaxAbs>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
@@ -434,13 +449,13 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
                 ok = range_quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, k, tile, refill,
                                                                                 local_bucket, scale_writer);
         } else {
-            constexpr bool NORM = MODE == kNorm;
+            constexpr bool NORM = MODE == kNorm, GIVEN = MODE == kGiven;
             if (tile < c.full_tiles)
-                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM>(sh, wv, a, c, k, tile, refill,
-                                                                               local_bucket, scale_writer);
+                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM, GIVEN>(sh, wv, a, c, k, tile, refill,
+                                                                                      local_bucket, scale_writer);
             else
-                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM>(sh, wv, a, c, k, tile, refill,
-                                                                                local_bucket, scale_writer);
+                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM, GIVEN>(sh, wv, a, c, k, tile, refill,
+                                                                                       local_bucket, scale_writer);
         }
     }
     if (!ok) {
@@ -867,6 +882,39 @@ cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, u
         case 7: return launch_norm_bits<7>(map, a, c, dtype, shuffle, timeouts, stream);
         case 8: return launch_norm_bits<8>(map, a, c, dtype, shuffle, timeouts, stream);
     }
+    return cudaErrorInvalidValue;
+}
+
+// ---- encode against a given scale on the TMA kernel: one long segment (= one bucket) per launch ----
+bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset)
+{
+    return n >= (1ull << 20) && n / 32 <= 0x7FFFFFFFull && (elem_offset & 7u) == 0 &&
+           (reinterpret_cast<uintptr_t>(grad) & 15u) == 0 && (reinterpret_cast<uintptr_t>(codes) & 15u) == 0;
+}
+
+cudaError_t launch_quantize_given_scale(const void* grad, uint64_t n, int bits, uint64_t seed, uint32_t* codes,
+                                        float* scale, int dtype, uint32_t worker, uint32_t step,
+                                        uint64_t elem_offset, cudaStream_t stream)
+{
+    QuantizeArgs a;
+    fill_args(a, grad, n, bits, 128 * 32, seed, codes, scale, worker, step, elem_offset);   // tiles of 128 rows
+    a.nbuckets = 1;
+    TmaQuantizeConsts c;
+    if (fill_tma_args(a, c, 128) != 128) return cudaErrorInvalidValue;
+    unsigned int* timeouts = wait_timeout_counter();
+    if (timeouts == nullptr) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const char* why = nullptr;
+    if (!encode_rows_map(&map, grad, a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why))
+        return cudaErrorNotSupported;
+#define MQG_GIVEN_CASE(B) \
+    case B: return dtype == 0 ? launch_tma_inst<B, 0, 128, false, kGiven>(map, a, c, timeouts, stream) \
+                              : launch_tma_inst<B, 1, 128, false, kGiven>(map, a, c, timeouts, stream)
+    switch (bits) {
+        MQG_GIVEN_CASE(1); MQG_GIVEN_CASE(2); MQG_GIVEN_CASE(3); MQG_GIVEN_CASE(4);
+        MQG_GIVEN_CASE(5); MQG_GIVEN_CASE(6); MQG_GIVEN_CASE(7); MQG_GIVEN_CASE(8);
+    }
+#undef MQG_GIVEN_CASE
     return cudaErrorInvalidValue;
 }
 

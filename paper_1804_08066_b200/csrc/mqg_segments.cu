@@ -139,16 +139,35 @@ static cudaError_t two_pass(const SegQuantArgs& a, const SegmentTable& tab, uint
     return launch_encode_segments(a, tab, bits, dtype, grid, stream);
 }
 
-cudaError_t launch_quantize_segments(const void* grad, const SegmentTable& tab, int bits,
-                                     uint64_t seed, uint32_t* codes, float* scales_base, int dtype,
-                                     uint32_t worker, uint32_t step, uint64_t elem_offset,
-                                     cudaStream_t stream)
+// The two passes of the per-layer quantizer as separate launches (the caller may give some segments'
+// encode to another kernel): the max pass over every segment of `tab`, and the encode pass over the
+// tiles `tab` lists.
+cudaError_t launch_segments_absmax(const void* grad, const SegmentTable& tab, float* scales_base, int dtype,
+                                   cudaStream_t stream)
+{
+    SegQuantArgs a;
+    a.grad = grad; a.codes = nullptr; a.scales = scales_base; a.elem_offset = 0;
+    a.key.seed_lo = a.key.seed_hi = a.key.worker = a.key.step = 0;
+    cudaError_t err = cudaMemsetAsync(scales_base, 0, (size_t)tab.nseg * sizeof(float), stream);
+    if (err != cudaSuccess) return err;
+    const uint32_t ntiles = tab.tile_start[tab.nseg];
+    if (ntiles == 0) return cudaSuccess;
+    if (dtype == 0) absmax_segments_kernel<0><<<ntiles, kMaxTileRows, 0, stream>>>(a, tab);
+    else absmax_segments_kernel<1><<<ntiles, kMaxTileRows, 0, stream>>>(a, tab);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_segments_encode(const void* grad, const SegmentTable& tab, int bits, uint64_t seed,
+                                   uint32_t* codes, float* scales_base, int dtype, uint32_t worker,
+                                   uint32_t step, uint64_t elem_offset, cudaStream_t stream)
 {
     SegQuantArgs a;
     a.grad = grad; a.codes = codes; a.scales = scales_base; a.elem_offset = elem_offset;
     a.key.seed_lo = (uint32_t)seed; a.key.seed_hi = (uint32_t)(seed >> 32);
     a.key.worker = worker; a.key.step = step;
-    return two_pass(a, tab, tab.tile_start[tab.nseg], (uint64_t)tab.nseg, bits, dtype, stream);
+    const uint32_t ntiles = tab.tile_start[tab.nseg];
+    if (ntiles == 0) return cudaSuccess;
+    return launch_encode_segments(a, tab, bits, dtype, ntiles, stream);
 }
 
 cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, uint64_t bucket,

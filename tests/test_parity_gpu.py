@@ -280,7 +280,7 @@ def test_segments_quantize_and_server(bits):
 
 
 @pytest.mark.parametrize("bits", [1, 3, 8])
-def test_segments_server_long_segments_take_their_own_launch(bits):
+def test_segments_long_segments_take_their_own_launches(bits):
     """Segments of a million elements and more go to the TMA-fed kernel when their buffers are
     16-byte aligned (the second one here, ragged length included) and stay in the table-driven
     launch otherwise (the fourth one starts on an odd word); both must match the checker."""
@@ -289,8 +289,21 @@ def test_segments_server_long_segments_take_their_own_launch(bits):
     seg, coff = _segments(sizes, bits)
     n = int(seg[-1])
     xs = [wl.layered(sizes, config=3, worker=w) for w in range(W)]
+    xs[1][128:128 + (1 << 20) + 37] = np.float32(1e-30)     # a long segment whose maximum is flushed to 0
     refs = [O.quantize_segments(x, seg, coff, bits, seed=5, worker=w) for w, x in enumerate(xs)]
     codes, scales = [r[0] for r in refs], [r[1] for r in refs]
+    for w in (0, 1):                                        # the quantizer routes long segments too
+        dc = Guarded(int(coff[-1]), torch.int32)
+        ds = Guarded(len(sizes), torch.float32)
+        mqg.mqg_quantize_segments(to_dev(xs[w]), seg, coff, bits, 5, dc.view, ds.view, worker=w)
+        torch.cuda.synchronize()
+        dc.check_guards(), ds.check_guards()
+        assert bits_equal(ds.numpy(np.float32), scales[w]) == 0
+        got = dc.numpy(np.uint32)
+        for j, sz in enumerate(sizes):
+            lo, nw = int(coff[j]), O.code_words(sz, bits)
+            assert np.array_equal(got[lo:lo + nw], codes[w][lo:lo + nw]), (w, j)
+    assert scales[1][1] == 0 and scales[0][1] > 0
     p0 = wl.params(n, 0.05, config=3)
     p_ref, _ = O.server_step_segments(codes, scales, bits, seg, coff, p0.copy(), 0.05)
     p = Guarded(n, torch.float32, fill=p0)

@@ -164,6 +164,17 @@ def test_segments_quantize(bits):
     segments_parity(sizes, bits, x, seed=3, worker=1, step=1, elem_offset=64)
 
 
+@pytest.mark.parametrize("bits", [3, 8])
+def test_segments_long_segments_encode_in_their_own_launches(bits):
+    """Segments of a million elements and more with 16-byte aligned buffers (the second one here,
+    ragged length included) are encoded by the TMA-fed kernel, the others (the fourth starts on an
+    odd word) by the table-driven launch; scales and codes must match the checker either way."""
+    sizes = [128, (1 << 20) + 37, 5, (1 << 20) + 64, 100]
+    x = wl.layered(sizes, config=3, worker=2)
+    x[128 + (1 << 20) + 37 + 5:128 + (1 << 20) + 37 + 5 + 4096] = 0.0
+    segments_parity(sizes, bits, x, seed=6, worker=2, step=1)
+
+
 def test_segments_more_than_one_launch_chunk_and_a_dirty_workspace():
     rng = np.random.default_rng(0)
     sizes = [int(v) for v in rng.integers(0, 30_000, 150)]
