@@ -649,7 +649,16 @@ def run_single_kernel(args):
     n, W, B, b = args.n, args.workers, args.bucket, args.bits
     rot = 3                                    # rotate buffer sets so launches never re-read L2
     stream = torch.cuda.current_stream()
-    if args.kernel == "quantize":
+    if args.kernel == "quantize" and args.dtype == "bf16":
+        # the stress shape's input type: heavy-tailed bf16 values widened in the kernel
+        grads = [torch.from_numpy(wl.student_t_bf16(n, config=5, worker=w).view(np.int16)).cuda().view(torch.bfloat16)
+                 for w in range(rot)]
+        codes = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
+        scales = [torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize(grads[i % rot], n, b, B, PHILOX_SEED, codes[i % rot],
+                                            scales[i % rot], worker=i % rot, step=i)
+        nbytes = quantize_bytes(n, b, B) - 2 * n
+    elif args.kernel == "quantize":
         grads = [torch.from_numpy(wl.laplace(n, LAPLACE_SCALE, config=2, worker=w)).cuda() for w in range(rot)]
         codes = [torch.zeros(mqg.mqg_code_words(n, b), dtype=torch.int32, device="cuda") for _ in range(rot)]
         scales = [torch.zeros(mqg.mqg_num_buckets(n, B), dtype=torch.float32, device="cuda") for _ in range(rot)]
@@ -768,6 +777,7 @@ def main():
                     default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--dtype", choices=["f32", "bf16"], default="f32", help="gradient type of --kernel quantize")
     ap.add_argument("--n", type=int, default=1 << 25)
     ap.add_argument("--workers", type=int, default=N_WORKERS)
     ap.add_argument("--bucket", type=int, default=BUCKET)
