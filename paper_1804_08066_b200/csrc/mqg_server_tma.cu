@@ -1,6 +1,6 @@
 // Fused server pass fed entirely by TMA (the fast path of mqg_server_step for uniform buckets of
-// at least 1024 elements): every WARP is an independent pipeline over a contiguous range of
-// 32-row tiles.  Nothing is loaded through registers:
+// at least 1024 elements, and of 512, 768, 896, 960 or 992): every WARP is an independent pipeline
+// over a contiguous range of 32-row tiles.  Nothing is loaded through registers:
 //   * a tile's 32 x 32 parameters arrive by a tiled bulk copy into the warp's own swizzled
 //     shared-memory stage (two stages, the next tile always in flight), are updated in place and
 //     leave by a tiled bulk store;
@@ -36,7 +36,7 @@ struct ServerTmaArgs {
     uint32_t nrows_full;         // floor(n / 32): rows the tensor map and the code copies cover
     uint32_t ntiles;             // ceil(nrows_full / 32)
     uint32_t nbuckets;
-    uint32_t rows_per_bucket;    // >= 32, so a tile touches at most two buckets
+    uint32_t rows_per_bucket;    // such that a tile touches at most two buckets (server_tma_applies)
     int rpb_shift;               // log2(rows_per_bucket) if a power of two, else -1
     int W;
     float neg_lr;
@@ -417,7 +417,16 @@ bool server_tma_applies(uint64_t n, uint64_t bucket)
 {
     const uint64_t nrows = (n + 31) / 32;
     const uint64_t rpb = bucket >= n ? nrows : bucket / 32;
-    return n / 32 >= 4 * (uint64_t)kSrvTileRows && nrows <= 0x7FFFFFFFull && rpb >= (uint64_t)kSrvTileRows;
+    if (n / 32 < 4 * (uint64_t)kSrvTileRows || nrows > 0x7FFFFFFFull) return false;
+    if (rpb >= (uint64_t)kSrvTileRows) return true;
+    // Shorter buckets qualify when no 32-row tile (tiles start at multiples of 32 rows) can hold two
+    // bucket boundaries, i.e. touch three buckets: the boundaries' offsets inside a tile are multiples
+    // of g = gcd(rows per bucket, 32), so the first one lies at least g rows in and the next one
+    // rows-per-bucket further: beyond the tile iff g + rpb >= 32 (buckets of 16, 24, 28, 30, 31 rows).
+    if (rpb < 16) return false;
+    uint64_t g = rpb, r = 32;
+    while (r != 0) { const uint64_t t = g % r; g = r; r = t; }
+    return g + rpb >= 32;
 }
 
 // mode 1: dst = params (update with lr); mode 0: dst = acc (overwrite); mode 2: dst = acc (add into)

@@ -171,7 +171,11 @@ def test_server_step_config1(bits):
 @pytest.mark.parametrize("bits", ALL_BITS)
 @pytest.mark.parametrize("n,bucket,W", [(1, 32, 1), (33, 32, 2), (8192 + 5, 2048, 3),
                                         (100_003, 4096, 5), (9000, 96, 2), (5000, 10_000, 4),
-                                        (3 * 32768 + 77, 32768, 2), (65_536 + 31, 512, 32)])
+                                        (3 * 32768 + 77, 32768, 2), (65_536 + 31, 512, 32),
+                                        # buckets shorter than a 32-row tile that still take the TMA-fed kernel
+                                        # (16, 24, 28, 30, 31 rows) and one that does not (20 rows)
+                                        (40_000 + 5, 768, 3), (50_000, 896, 2), (33_333, 960, 2),
+                                        (70_001, 992, 3), (30_000, 640, 2)])
 def test_server_step_shapes(bits, n, bucket, W):
     xs = [wl.normal(n, 2e-3, config=21, worker=w) for w in range(W)]
     xs[0][: min(n, 40)] = 0.0
