@@ -105,7 +105,8 @@ cudaError_t launch_server(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, u
 
 // TMA-fed server pass over uniform buckets of >= 32 rows.  mode 1: dst = params, updated with lr;
 // mode 0: dst = acc, overwritten with the sum; mode 2: dst = acc, the sum continues from it.
-bool server_tma_applies(uint64_t n, uint64_t bucket);
+bool server_tma_applies(uint64_t n, uint64_t bucket);          // for any worker count
+bool server_tma_applies(uint64_t n, uint64_t bucket, int W);   // also buckets of 32 .. 256 elements for few workers
 cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                               float* dst, float lr, int mode, cudaStream_t stream);
 

@@ -224,7 +224,7 @@ range_server_kernel(const __grid_constant__ RangeServerArgs a)
 cudaError_t launch_server_range(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                                 float* params, float lr, float* acc, int add_into, cudaStream_t stream)
 {
-    if (server_tma_applies(n, bucket)) {
+    if (server_tma_applies(n, bucket, W)) {
         if (params != nullptr && acc == nullptr)
             return launch_server_range_tma(ptrs, W, bits, n, bucket, params, lr, 1, stream);
         if (params == nullptr)

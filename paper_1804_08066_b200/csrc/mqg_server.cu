@@ -170,7 +170,7 @@ static cudaError_t dispatch_bits(int bits, const ServerArgs& a, const SegmentTab
 cudaError_t launch_server(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                           float* params, float lr, float* acc, int add_into, cudaStream_t stream)
 {
-    if (server_tma_applies(n, bucket)) {
+    if (server_tma_applies(n, bucket, W)) {
         if (params != nullptr && acc == nullptr)
             return launch_server_tma(ptrs, W, bits, n, bucket, params, lr, 1, stream);
         if (params == nullptr)

@@ -1,5 +1,6 @@
 // Fused server pass fed entirely by TMA (the fast path of mqg_server_step for uniform buckets of
-// at least 1024 elements, and of 512, 768, 896, 960 or 992): every WARP is an independent pipeline
+// at least 1024 elements, of 512, 768, 896, 960 or 992, and - for few workers - of 32 to 256): every
+// WARP is an independent pipeline
 // over a contiguous range of 32-row tiles.  Nothing is loaded through registers:
 //   * a tile's 32 x 32 parameters arrive by a tiled bulk copy into the warp's own swizzled
 //     shared-memory stage (two stages, the next tile always in flight), are updated in place and
@@ -36,8 +37,10 @@ struct ServerTmaArgs {
     uint32_t nrows_full;         // floor(n / 32): rows the tensor map and the code copies cover
     uint32_t ntiles;             // ceil(nrows_full / 32)
     uint32_t nbuckets;
-    uint32_t rows_per_bucket;    // such that a tile touches at most two buckets (server_tma_applies)
+    uint32_t rows_per_bucket;    // such that a tile touches at most 1 << nbt_shift buckets
     int rpb_shift;               // log2(rows_per_bucket) if a power of two, else -1
+    int nbt_shift;               // log2 of the buckets a tile can touch: 1 (two buckets), or 2..5 for
+                                 // buckets of 8, 4, 2, 1 rows; W << nbt_shift <= 2 * kMaxWorkers
     int W;
     float neg_lr;
     uint32_t bias_bits;          // 0x4B000000 (2^23), a run-time constant for the byte permutes
@@ -48,7 +51,8 @@ template <int BITS>
 struct ServerSmem {
     alignas(1024) uint8_t stage[kSrvWarps][2][kSrvTileBytes];
     alignas(16) uint32_t code[kSrvWarps][kCodeDepth][ServerGroup<BITS>::value][kSrvTileRows * BITS];
-    float2 table[kSrvWarps][2][kMaxWorkers][2];   // (2h, -h) per worker and bucket of the tile
+    float2 table[kSrvWarps][2][2 * kMaxWorkers];  // (2h, -h) per (worker, bucket of the tile): entry
+                                                  // (worker << nbt_shift) + bucket-of-tile
     uint64_t bar[kSrvWarps][2];                   // parameter stages
     uint64_t cbar[kSrvWarps][kCodeDepth];         // code stages
 };
@@ -68,7 +72,8 @@ __device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_
     const uint32_t first = bucket_of_row(a, row0);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const uint32_t pair = lane + 32u * h, w = pair >> 1, b = first + (pair & 1u);
+        const uint32_t pair = lane + 32u * h, w = pair >> a.nbt_shift;
+        const uint32_t b = first + (pair & ((1u << a.nbt_shift) - 1u));
         const bool have = w < (uint32_t)a.W && b < a.nbuckets;
         if (RANGE) s[h] = have ? __ldg(reinterpret_cast<const float2*>(a.ptrs.scales[w]) + b) : make_float2(0.0f, 0.0f);
         else s[h] = make_float2(have ? __ldg(a.ptrs.scales[w] + b) : 0.0f, 0.0f);
@@ -76,15 +81,15 @@ __device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_
 }
 
 template <int BITS, bool RANGE>
-__device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float2 (*table)[2], uint32_t lane,
+__device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float2* table, uint32_t lane,
                                                   const float2 (&s)[2])
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const uint32_t pair = lane + 32u * h, w = pair >> 1;
+        const uint32_t pair = lane + 32u * h, w = pair >> a.nbt_shift;
         if (w < (uint32_t)a.W) {
             const DecodeScale d = RANGE ? range_decode_scale<BITS>(s[h].x, s[h].y) : decode_scale<BITS>(s[h].x);
-            table[w][pair & 1u] = make_float2(d.two_h, d.minus_h);
+            table[pair] = make_float2(d.two_h, d.minus_h);
         }
     }
 }
@@ -267,7 +272,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
             auto decode_worker = [&](int i) {
                 uint32_t w[BITS];
                 read_stage_words<BITS>(cstage + i * (kSrvTileRows * BITS) + lane * BITS, w);
-                const float2 e = sm.table[wid][stg][g0 + i][lb];
+                const float2 e = sm.table[wid][stg][((uint32_t)(g0 + i) << a.nbt_shift) + lb];
                 DecodeScale2 d;
                 d.two_h = make_float2(e.x, e.x); d.minus_h = make_float2(e.y, e.y);
                 add_decoded_row<BITS, RANGE>(w, d, v2, a.bias_bits);
@@ -429,6 +434,22 @@ bool server_tma_applies(uint64_t n, uint64_t bucket)
     return g + rpb >= 32;
 }
 
+// log2 of the buckets a tile can touch, or -1 if the kernel does not take the shape: 1 for the shapes
+// above; buckets of 8, 4, 2 or 1 rows (256 .. 32 elements) divide a tile into 4 .. 32 buckets, which
+// the warp's table of 2 * kMaxWorkers entries holds for up to 16, 8, 4, 2 workers.
+static int server_tma_nbt_shift(uint64_t n, uint64_t bucket, int W)
+{
+    if (server_tma_applies(n, bucket)) return 1;
+    const uint64_t nrows = (n + 31) / 32;
+    if (n / 32 < 4 * (uint64_t)kSrvTileRows || nrows > 0x7FFFFFFFull || bucket >= n) return -1;
+    const uint64_t rpb = bucket / 32;
+    for (int sft = 2; sft <= 5; ++sft)
+        if (rpb == (32u >> sft)) return ((uint64_t)W << sft) <= 2 * (uint64_t)kMaxWorkers ? sft : -1;
+    return -1;
+}
+
+bool server_tma_applies(uint64_t n, uint64_t bucket, int W) { return server_tma_nbt_shift(n, bucket, W) >= 0; }
+
 // mode 1: dst = params (update with lr); mode 0: dst = acc (overwrite); mode 2: dst = acc (add into)
 template <bool RANGE>
 static cudaError_t launch_server_tma_codec(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
@@ -448,6 +469,8 @@ static cudaError_t launch_server_tma_codec(const WorkerPtrs& ptrs, int W, int bi
     a.rpb_shift = -1;
     for (int sft = 0; sft < 32; ++sft)
         if (((uint64_t)1 << sft) == rpb) a.rpb_shift = sft;
+    a.nbt_shift = server_tma_nbt_shift(n, bucket, W);
+    if (a.nbt_shift < 0) return cudaErrorInvalidValue;
     a.W = W;
     a.neg_lr = -lr;
     a.bias_bits = 0x4B000000u;

@@ -175,7 +175,10 @@ def test_server_step_config1(bits):
                                         # buckets shorter than a 32-row tile that still take the TMA-fed kernel
                                         # (16, 24, 28, 30, 31 rows) and one that does not (20 rows)
                                         (40_000 + 5, 768, 3), (50_000, 896, 2), (33_333, 960, 2),
-                                        (70_001, 992, 3), (30_000, 640, 2)])
+                                        (70_001, 992, 3), (30_000, 640, 2),
+                                        # buckets of 8, 4, 2, 1 rows: TMA-fed for few workers, else the general kernel
+                                        (50_000 + 3, 256, 8), (50_000, 256, 20), (40_000 + 7, 128, 8),
+                                        (40_000, 64, 4), (30_000, 32, 2), (30_000 + 1, 32, 3)])
 def test_server_step_shapes(bits, n, bucket, W):
     xs = [wl.normal(n, 2e-3, config=21, worker=w) for w in range(W)]
     xs[0][: min(n, 40)] = 0.0

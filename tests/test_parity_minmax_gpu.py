@@ -98,6 +98,7 @@ def encode_workers(xs, bits, bucket):
     (40_000, 96, 2),            # small buckets: the general kernel
     (33, 32, 2), (1, 32, 1),
     (70_000, 1 << 20, 5),       # a single bucket
+    (50_000 + 3, 512, 6), (40_000 + 5, 768, 3), (50_000, 256, 8), (40_000 + 7, 128, 3), (30_000, 32, 2),
 ])
 def test_server_step_and_accumulate(bits, n, bucket, W):
     xs = [wl.laplace(n, 10.0 ** (-3 + (w % 3)), config=2, worker=w) for w in range(W)]
