@@ -1,7 +1,7 @@
 // Fused server pass fed entirely by TMA (the fast path of mqg_server_step for uniform buckets of
 // at least 1024 elements, of 512, 768, 896, 960 or 992, and - for few workers - of 32 to 256): every
-// WARP is an independent pipeline
-// over a contiguous range of 32-row tiles.  Nothing is loaded through registers:
+// WARP is an independent pipeline over a contiguous range of 32-row tiles.  Nothing is loaded
+// through registers:
 //   * a tile's 32 x 32 parameters arrive by a tiled bulk copy into the warp's own swizzled
 //     shared-memory stage (two stages, the next tile always in flight), are updated in place and
 //     leave by a tiled bulk store;
