@@ -25,11 +25,35 @@ struct RequantArgs {
 // the tile holds at most kTableBuckets buckets; smaller buckets compute them per row.
 constexpr int kTableBuckets = 32;
 
+// A row's BITS words from a staged copy of a worker's code words (widest access the offset allows).
+template <int BITS>
+__device__ __forceinline__ void staged_row_words(const uint32_t* __restrict__ p, uint32_t (&w)[BITS])
+{
+    if constexpr (BITS % 4 == 0) {
+#pragma unroll
+        for (int k = 0; k < BITS / 4; ++k) {
+            const uint4 v = reinterpret_cast<const uint4*>(p)[k];
+            w[4 * k] = v.x; w[4 * k + 1] = v.y; w[4 * k + 2] = v.z; w[4 * k + 3] = v.w;
+        }
+    } else if constexpr (BITS % 2 == 0) {
+#pragma unroll
+        for (int k = 0; k < BITS / 2; ++k) {
+            const uint2 v = reinterpret_cast<const uint2*>(p)[k];
+            w[2 * k] = v.x; w[2 * k + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < BITS; ++k) w[k] = p[k];
+    }
+}
+
 // One tile.  FULL: every thread owns a complete row (vector loads, no bounds checks).  TABLE: the
-// de-quantization constants come from the shared table.
-template <int BITS, bool FULL, bool TABLE>
+// de-quantization constants come from the shared table.  STAGE (full tiles only): all workers' code
+// words of the tile are copied into shared memory by 16-byte asynchronous copies at the start, so
+// that no worker's decode waits for a global load.
+template <int BITS, bool FULL, bool TABLE, bool STAGE>
 __device__ __forceinline__ void requantize_tile(const RequantArgs& a, uint32_t* s_bucket,
-                                                float2 (*s_table)[kTableBuckets])
+                                                float2 (*s_table)[kTableBuckets], uint32_t* s_codes)
 {
     const uint32_t t = threadIdx.x;
     const uint64_t row0 = (uint64_t)blockIdx.x * a.tile_rows;
@@ -40,6 +64,14 @@ __device__ __forceinline__ void requantize_tile(const RequantArgs& a, uint32_t* 
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const uint64_t bucket = (uint64_t)blockIdx.x * a.buckets_per_tile + local_bucket;
 
+    constexpr uint32_t kWorkerWords = kMaxTileRows * BITS;      // one worker's words of a full tile
+    if constexpr (FULL && STAGE) {
+        const uint32_t chunks = (uint32_t)a.W * (kWorkerWords / 4);
+        for (uint32_t idx = t; idx < chunks; idx += kMaxTileRows) {
+            const uint32_t w = idx / (kWorkerWords / 4), c = idx - w * (kWorkerWords / 4);
+            cp_async16(s_codes + w * kWorkerWords + 4 * c, a.ptrs.codes[w] + row0 * BITS + 4 * c);
+        }
+    }
     if (t < a.buckets_per_tile) s_bucket[t] = 0u;
     if (TABLE) {
         for (uint32_t idx = t; idx < (uint32_t)a.W * a.buckets_per_tile; idx += blockDim.x) {
@@ -49,6 +81,7 @@ __device__ __forceinline__ void requantize_tile(const RequantArgs& a, uint32_t* 
             s_table[w][lbk] = make_float2(d.two_h, d.minus_h);
         }
     }
+    if constexpr (FULL && STAGE) cp_async_wait_all();
     __syncthreads();
 
     float x[32];
@@ -60,7 +93,9 @@ __device__ __forceinline__ void requantize_tile(const RequantArgs& a, uint32_t* 
 #pragma unroll 4
         for (int w = 0; w < a.W; ++w) {
             uint32_t cw[BITS];
-            if (FULL) {
+            if constexpr (FULL && STAGE) {
+                staged_row_words<BITS>(s_codes + w * kWorkerWords + t * BITS, cw);
+            } else if (FULL) {
                 load_row_words<BITS>(a.ptrs.codes[w], word0, cw);
             } else {
 #pragma unroll
@@ -122,21 +157,50 @@ __device__ __forceinline__ void requantize_tile(const RequantArgs& a, uint32_t* 
     }
 }
 
-template <int BITS, bool TABLE>
+template <int BITS, bool TABLE, bool STAGE>
 __global__ void __launch_bounds__(kMaxTileRows)
 requantize_kernel(const __grid_constant__ RequantArgs a)
 {
+    extern __shared__ __align__(16) uint32_t s_codes[];        // STAGE: W x 256 x BITS words
     __shared__ uint32_t s_bucket[kMaxTileRows];
     __shared__ float2 s_table[TABLE ? kMaxWorkers : 1][kTableBuckets];
-    if (blockIdx.x < a.full_tiles) requantize_tile<BITS, true, TABLE>(a, s_bucket, s_table);
-    else requantize_tile<BITS, false, TABLE>(a, s_bucket, s_table);
+    if (blockIdx.x < a.full_tiles) requantize_tile<BITS, true, TABLE, STAGE>(a, s_bucket, s_table, s_codes);
+    else requantize_tile<BITS, false, TABLE, STAGE>(a, s_bucket, s_table, s_codes);
 }
 
+// Code words are staged in shared memory when all workers' words of a tile fit in 64 KB (three CTAs
+// per SM at that size; the kernel is bound by arithmetic, not by occupancy).
+constexpr size_t kMaxStagedCodeBytes = 64 * 1024;
+
 template <int BITS>
-static void launch_requantize_bits(const RequantArgs& a, unsigned grid, cudaStream_t stream)
+static cudaError_t launch_requantize_bits(const RequantArgs& a, unsigned grid, cudaStream_t stream)
 {
-    if (a.buckets_per_tile <= (uint32_t)kTableBuckets) requantize_kernel<BITS, true><<<grid, kMaxTileRows, 0, stream>>>(a);
-    else requantize_kernel<BITS, false><<<grid, kMaxTileRows, 0, stream>>>(a);
+    if (a.buckets_per_tile > (uint32_t)kTableBuckets) {
+        requantize_kernel<BITS, false, false><<<grid, kMaxTileRows, 0, stream>>>(a);
+        return cudaGetLastError();
+    }
+    // Measured per width at n = 25 M, W = 8 (us per launch, register loads -> staged): 2: 60.6 -> 51.9,
+    // 3: 58.4 -> 54.5, 4: 58.6 -> 57.0, 8: 67.9 -> 57.5; 1 unchanged; 5, 6, 7 two microseconds slower
+    // (their rows are not 8- or 16-byte multiples, so the staged words are read back one by one).
+    constexpr bool kStagePays = BITS == 2 || BITS == 3 || BITS == 4 || BITS == 8;
+    const size_t staged = (size_t)a.W * kMaxTileRows * BITS * sizeof(uint32_t);
+    if (!kStagePays || a.full_tiles == 0 || staged > kMaxStagedCodeBytes) {
+        requantize_kernel<BITS, true, false><<<grid, kMaxTileRows, 0, stream>>>(a);
+        return cudaGetLastError();
+    }
+    static bool configured[64] = {};                           // per device
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        err = cudaFuncSetAttribute(requantize_kernel<BITS, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)kMaxStagedCodeBytes);
+        if (err != cudaSuccess) return err;
+        configured[dev] = true;
+    }
+    requantize_kernel<BITS, true, true><<<grid, kMaxTileRows, staged, stream>>>(a);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
@@ -166,17 +230,16 @@ cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
     a.full_tiles = a.tile_rows == (uint32_t)kMaxTileRows ? (uint32_t)((n / 32) / a.tile_rows) : 0u;
     const unsigned grid = (unsigned)ntiles;
     switch (bits) {
-        case 1: launch_requantize_bits<1>(a, grid, stream); break;
-        case 2: launch_requantize_bits<2>(a, grid, stream); break;
-        case 3: launch_requantize_bits<3>(a, grid, stream); break;
-        case 4: launch_requantize_bits<4>(a, grid, stream); break;
-        case 5: launch_requantize_bits<5>(a, grid, stream); break;
-        case 6: launch_requantize_bits<6>(a, grid, stream); break;
-        case 7: launch_requantize_bits<7>(a, grid, stream); break;
-        case 8: launch_requantize_bits<8>(a, grid, stream); break;
-        default: return cudaErrorInvalidValue;
+        case 1: return launch_requantize_bits<1>(a, grid, stream);
+        case 2: return launch_requantize_bits<2>(a, grid, stream);
+        case 3: return launch_requantize_bits<3>(a, grid, stream);
+        case 4: return launch_requantize_bits<4>(a, grid, stream);
+        case 5: return launch_requantize_bits<5>(a, grid, stream);
+        case 6: return launch_requantize_bits<6>(a, grid, stream);
+        case 7: return launch_requantize_bits<7>(a, grid, stream);
+        case 8: return launch_requantize_bits<8>(a, grid, stream);
     }
-    return cudaGetLastError();
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace mqg
