@@ -1,13 +1,17 @@
-// Fused server pass fed entirely by TMA (the fast path of mqg_server_step for uniform buckets of
-// at least 1024 elements, of 512, 768, 896, 960 or 992, and - for few workers - of 32 to 256): every
-// WARP is an independent pipeline over a contiguous range of 32-row tiles.  Nothing is loaded
-// through registers:
-//   * a tile's 32 x 32 parameters arrive by a tiled bulk copy into the warp's own swizzled
-//     shared-memory stage (two stages, the next tile always in flight), are updated in place and
-//     leave by a tiled bulk store;
+// Fused server pass (the fast path of mqg_server_step for uniform buckets of at least 1024 elements,
+// of 512, 768, 896, 960 or 992, and - for few workers - of 32 to 256): every WARP is an independent
+// pipeline over a contiguous range of 32-row tiles.  Nothing is loaded through registers:
+//   * a tile's 32 x 32 parameters arrive by a tiled bulk copy (TMA) into the warp's own swizzled
+//     shared-memory stage while the tile's workers are being summed, are updated in place and leave
+//     by a tiled bulk store;
 //   * the code words of the tile (32 rows x K words per worker, contiguous in each worker's
-//     stream) arrive by one linear bulk copy per worker into a two-deep ring of code stages, a
-//     group of workers per stage, issued two stages ahead of their use.
+//     stream) arrive by 16-byte asynchronous copies, one instruction of the warp per worker (two
+//     above four bits), into a two-deep ring of code stages, a group of workers per stage, issued
+//     two stages ahead of their use.  (One linear bulk copy per worker, completing on an mbarrier,
+//     cost about a dozen instructions of the warp per copy - the operands of a bulk copy travel
+//     through the uniform datapath - and with eight of them per tile a third of the kernel's
+//     instructions were overhead: 40.1 executed instructions per parameter at four bits and eight
+//     workers against 31.4 now.)
 // A warp therefore never waits for DRAM latency in steady state and there is no CTA-wide barrier
 // anywhere.  Per-(worker, bucket) de-quantization constants are computed once per tile into the
 // warp's small shared table, one tile ahead.
@@ -23,11 +27,11 @@ constexpr int kSrvTileRows = 32;                  // rows per tile = lanes per w
 constexpr uint32_t kSrvTileBytes = kSrvTileRows * 128;
 constexpr int kCodeDepth = 2;                     // code stages per warp
 
-// Workers whose code words share one code stage: at most 2 KB per stage, so that a CTA's shared
+// Workers whose code words share one code stage: at most 4 KB per stage, so that a CTA's shared
 // memory (13 KB per warp) lets four CTAs = 16 warps share an SM, and a power of two, so that the
 // usual worker counts fill whole stages.
 template <int BITS>
-struct ServerGroup { static constexpr int value = BITS <= 2 ? 8 : (BITS <= 4 ? 4 : 2); };
+struct ServerGroup { static constexpr int value = BITS <= 4 ? 8 : 4; };
 
 struct ServerTmaArgs {
     WorkerPtrs ptrs;
@@ -44,17 +48,17 @@ struct ServerTmaArgs {
     int W;
     float neg_lr;
     uint32_t bias_bits;          // 0x4B000000 (2^23), a run-time constant for the byte permutes
+    uint32_t poll_limit;         // polls of one barrier wait before the warp gives up
 };
 
 // Dynamic shared memory of one CTA (base rounded up to 1024 bytes for the 128-byte swizzle).
 template <int BITS>
 struct ServerSmem {
-    alignas(1024) uint8_t stage[kSrvWarps][2][kSrvTileBytes];
+    alignas(1024) uint8_t stage[kSrvWarps][kSrvTileBytes];      // one parameter tile per warp
     alignas(16) uint32_t code[kSrvWarps][kCodeDepth][ServerGroup<BITS>::value][kSrvTileRows * BITS];
-    float2 table[kSrvWarps][2][2 * kMaxWorkers];  // (2h, -h) per (worker, bucket of the tile): entry
+    float4 table[kSrvWarps][2 * kMaxWorkers];     // (2h, 2h, -h, -h) per (worker, bucket of the tile): entry
                                                   // (worker << nbt_shift) + bucket-of-tile
-    uint64_t bar[kSrvWarps][2];                   // parameter stages
-    uint64_t cbar[kSrvWarps][kCodeDepth];         // code stages
+    uint64_t bar[kSrvWarps];                      // parameter tile landed
 };
 
 __device__ __forceinline__ uint32_t bucket_of_row(const ServerTmaArgs& a, uint32_t row)
@@ -62,16 +66,18 @@ __device__ __forceinline__ uint32_t bucket_of_row(const ServerTmaArgs& a, uint32
     return a.rpb_shift >= 0 ? row >> a.rpb_shift : row / a.rows_per_bucket;
 }
 
-// Scales of the (worker, bucket) pairs of the tile that starts at row0: lane l holds pair l and
-// pair l + 32 (pair = 2 * worker + bucket-of-tile).  RANGE: the pair's (lo, hi) instead of its
-// scale (the `scales` pointers then address arrays of two floats per bucket).
+// Scales of the (worker, bucket) pairs of the tile that starts at row0: lane l holds pair l and,
+// when there are more than 32 pairs (`wide`), pair l + 32 (pair = (worker << nbt_shift) +
+// bucket-of-tile).  RANGE: the pair's (lo, hi) instead of its scale (the `scales` pointers then
+// address arrays of two floats per bucket).
 template <bool RANGE>
 __device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_t row0, uint32_t lane,
-                                                 float2 (&s)[2])
+                                                 bool wide, float2 (&s)[2])
 {
     const uint32_t first = bucket_of_row(a, row0);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !wide) break;
         const uint32_t pair = lane + 32u * h, w = pair >> a.nbt_shift;
         const uint32_t b = first + (pair & ((1u << a.nbt_shift) - 1u));
         const bool have = w < (uint32_t)a.W && b < a.nbuckets;
@@ -81,15 +87,16 @@ __device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_
 }
 
 template <int BITS, bool RANGE>
-__device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float2* table, uint32_t lane,
-                                                  const float2 (&s)[2])
+__device__ __forceinline__ void store_tile_scales(const ServerTmaArgs& a, float4* table, uint32_t lane,
+                                                  bool wide, const float2 (&s)[2])
 {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !wide) break;
         const uint32_t pair = lane + 32u * h, w = pair >> a.nbt_shift;
         if (w < (uint32_t)a.W) {
             const DecodeScale d = RANGE ? range_decode_scale<BITS>(s[h].x, s[h].y) : decode_scale<BITS>(s[h].x);
-            table[pair] = make_float2(d.two_h, d.minus_h);
+            table[pair] = make_float4(d.two_h, d.two_h, d.minus_h, d.minus_h);
         }
     }
 }
@@ -119,41 +126,64 @@ __device__ __forceinline__ void read_stage_words(const uint32_t* __restrict__ st
     }
 }
 
+// 16-byte asynchronous copy that reads only the first `src_bytes` bytes of the source and fills the
+// rest of the 16 bytes with zeros.
+__device__ __forceinline__ void cp_async16_partial(uint32_t smem_dst, const void* gmem_src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gmem_src), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async16_to(uint32_t smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // Starts the copies of one code stage: the words of rows [row0, row0 + 32) (fewer in the last tile
 // of the gradient) of workers g0 .. g0 + group - 1 (those that exist).  A worker's words of these
-// rows are contiguous in its stream and start on a 16-byte boundary (row0 is a multiple of 32),
-// so each worker is one linear bulk copy; a last tile whose byte count is not a multiple of 16
-// is filled with ordinary loads and stores instead.  Called by the whole warp.
+// rows are contiguous in its stream and start on a 16-byte boundary (row0 is a multiple of 32):
+// the warp copies them in 16-byte pieces, lane l the l-th piece (and the (l + 32)-th for more than
+// four bits), asynchronously and without passing through registers.  The piece that holds the end
+// of a short last tile is copied up to that end and zero-filled.  `lane_off` = 16 * lane.
 template <int BITS>
-__device__ __forceinline__ void fill_code_stage(const ServerTmaArgs& a, uint32_t* stage, uint32_t bar,
-                                                uint32_t row0, int g0, uint32_t lane)
+__device__ __forceinline__ void fill_code_stage(const ServerTmaArgs& a, uint32_t stage, uint32_t row0, int g0,
+                                                uint32_t lane_off)
 {
     constexpr int kGroup = ServerGroup<BITS>::value;
-    constexpr uint32_t kWorkerWords = kSrvTileRows * BITS;
+    constexpr uint32_t kWorkerBytes = kSrvTileRows * BITS * 4;
+    constexpr int kPieces = (int)((kWorkerBytes / 16 + 31) / 32);       // pieces per lane: 1 or 2
     const uint32_t rows_here = min((uint32_t)kSrvTileRows, a.nrows_full - row0);
-    const int nwk = min(kGroup, a.W - g0);
-    const uint64_t word0 = (uint64_t)row0 * BITS;
-    if ((rows_here & 3u) == 0) {
-        if (lane == 0) {
-            const uint32_t bytes = rows_here * BITS * 4u;
-            mbar_expect_tx(bar, bytes * (uint32_t)nwk);
-            for (int i = 0; i < nwk; ++i)
-                bulk_load_1d(smem_u32(stage + i * kWorkerWords), a.ptrs.codes[g0 + i] + word0, bytes, bar);
-        }
-    } else {
-        if (lane < rows_here) {
-            for (int i = 0; i < nwk; ++i) {
-                const uint32_t* src = a.ptrs.codes[g0 + i] + word0 + lane * BITS;
+    const uint64_t byte0 = (uint64_t)row0 * (BITS * 4) + lane_off;
+    if (rows_here == (uint32_t)kSrvTileRows && g0 + kGroup <= a.W) {
 #pragma unroll
-                for (int j = 0; j < BITS; ++j) stage[i * kWorkerWords + lane * BITS + j] = __ldg(src + j);
+        for (int pc = 0; pc < kPieces; ++pc) {
+            if (lane_off + 512u * pc < kWorkerBytes) {
+#pragma unroll
+                for (int i = 0; i < kGroup; ++i)
+                    cp_async16_to(stage + i * kWorkerBytes + lane_off + 512u * pc,
+                                  reinterpret_cast<const uint8_t*>(a.ptrs.codes[g0 + i]) + byte0 + 512u * pc);
             }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar);
+    } else {
+        const uint32_t bytes_here = rows_here * BITS * 4;
+        const int nwk = min(kGroup, a.W - g0);
+#pragma unroll
+        for (int pc = 0; pc < kPieces; ++pc) {
+            const uint32_t off = lane_off + 512u * pc;
+            if (off < bytes_here) {
+                const uint32_t nb = min(16u, bytes_here - off);
+                for (int i = 0; i < nwk; ++i)
+                    cp_async16_partial(stage + i * kWorkerBytes + off,
+                                       reinterpret_cast<const uint8_t*>(a.ptrs.codes[g0 + i]) + byte0 + 512u * pc, nb);
+            }
+        }
     }
 }
 
-// CTAs per SM the register budget is set for (what the shared memory allows).
+// CTAs per SM the register budget is set for (what the shared memory allows at three bits and more;
+// five CTAs of 96 registers at one and two bits measured 0.3 us slower per launch than four).
 template <int BITS>
 constexpr int server_min_ctas() { return 4; }
 
@@ -169,20 +199,23 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     ServerSmem<BITS>& sm = *reinterpret_cast<ServerSmem<BITS>*>(
         smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     constexpr int kGroup = ServerGroup<BITS>::value;
-    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
-    uint8_t (*stage)[kSrvTileBytes] = sm.stage[wid];
-    uint64_t* bar = sm.bar[wid];
-    uint64_t* cbar = sm.cbar[wid];
+    constexpr uint32_t kWorkerWords = kSrvTileRows * BITS;
+    const uint32_t lane = threadIdx.x & 31u;
+    // the warp's number, taken from lane 0 so that the compiler knows it is the same in every lane
+    const uint32_t wid = __shfl_sync(0xFFFFFFFFu, threadIdx.x >> 5, 0);
+    uint8_t* stage = sm.stage[wid];
+    float4* table = sm.table[wid];
+    const uint32_t bar = smem_u32(&sm.bar[wid]);
+    const uint32_t code_base = smem_u32(&sm.code[wid][0][0][0]);
+    constexpr uint32_t kCodeStageBytes = kGroup * kWorkerWords * 4;
 
     if (lane == 0) {
-        mbar_init(smem_u32(&bar[0]), 1);
-        mbar_init(smem_u32(&bar[1]), 1);
-#pragma unroll
-        for (int s = 0; s < kCodeDepth; ++s) mbar_init(smem_u32(&cbar[s]), 1);
+        mbar_init(bar, 1);
         fence_barrier_init();
         prefetch_tensormap(&map_full);
     }
     __syncwarp();
+    grid_dependency_wait();            // nothing above touches global memory
 
     // this warp's tiles: [t_begin, t_begin + ntiles), the grid's tiles split evenly; the warps of the
     // first CTAs take the odd tiles (they start first; spreading the odd tiles evenly over the grid
@@ -195,21 +228,33 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     const uint32_t last_row = a.nrows_full - 1;    // nrows_full >= 1 on this path
     const uint32_t groups = ((uint32_t)a.W + kGroup - 1) / kGroup;      // code stages per tile
     const uint32_t nunits = ntiles * groups;
+    const bool wide = ((uint32_t)a.W << a.nbt_shift) > 32u;             // more than 32 table entries
+    const uint32_t lane_off = lane * 16u;
+    // MODE 1: the tile's parameters are requested before this worker of the tile is summed (see
+    // load_params below); measured best of 1 .. 4 at eight workers, per launch of n = 25 M: 55.8 us
+    // against 57.7 us at five bits, 65.2 against 68.0 us at eight, no difference up to four bits
+    constexpr int kIssueAt = 4;
+    const int issue_at = min(kIssueAt, a.W - 1);
 
     bool failed = false;
     uint32_t k = 0, u = 0;                         // tile and code stage in use
     if (ntiles > 0) {
         float2 s0[2];
-        load_tile_scales<RANGE>(a, r_begin, lane, s0);
-        store_tile_scales<BITS, RANGE>(a, sm.table[wid][0], lane, s0);
-        if (MODE != 0 && lane == 0) {
-            mbar_expect_tx(smem_u32(&bar[0]), kSrvTileBytes);
-            tma_load_2d(smem_u32(stage[0]), &map_full, 0, (int)r_begin, smem_u32(&bar[0]));
+        load_tile_scales<RANGE>(a, r_begin, lane, wide, s0);
+        store_tile_scales<BITS, RANGE>(a, table, lane, wide, s0);
+        if (MODE == 2 && lane == 0) {
+            mbar_expect_tx(bar, kSrvTileBytes);
+            tma_load_2d(smem_u32(stage), &map_full, 0, (int)r_begin, bar);
         }
-        // the first kCodeDepth code stages (u2 = stage number, tile u2 / groups, group u2 % groups)
-        for (uint32_t u2 = 0; u2 < (uint32_t)kCodeDepth && u2 < nunits; ++u2)
-            fill_code_stage<BITS>(a, &sm.code[wid][u2][0][0], smem_u32(&cbar[u2]),
-                                  r_begin + (u2 / groups) * kSrvTileRows, (int)(u2 % groups) * kGroup, lane);
+        // the first kCodeDepth code stages (u2 = stage number, tile u2 / groups, group u2 % groups);
+        // one copy group per stage, empty when there is no such stage
+#pragma unroll
+        for (uint32_t u2 = 0; u2 < (uint32_t)kCodeDepth; ++u2) {
+            if (u2 < nunits)
+                fill_code_stage<BITS>(a, code_base + u2 * kCodeStageBytes,
+                                      r_begin + (u2 / groups) * kSrvTileRows, (int)(u2 % groups) * kGroup, lane_off);
+            cp_async_commit();
+        }
         __syncwarp();
     }
     // position of the code stage kCodeDepth ahead of the one in use, kept incrementally
@@ -217,39 +262,26 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
 
 #pragma unroll 1
     for (; k < ntiles; ++k) {
-        const uint32_t stg = k & 1, parity = (k >> 1) & 1;
+        const uint32_t parity = k & 1;
         const uint32_t row0 = r_begin + k * kSrvTileRows;
         const bool have_next = k + 1 < ntiles;
-        // The other stage held tile k-1, whose store was committed at the end of the last
-        // iteration: once that store has read its source the stage can take tile k+1.
-        if (MODE == 0) {
-            // nothing is loaded: the stage is only written by this warp, once the store that used
-            // it two tiles ago has read it
-            if (lane == 0) bulk_wait_read<1>();
-            __syncwarp();
-        } else if (lane == 0 && have_next) {
-            bulk_wait_read<0>();
-            // the gradient's last tile may be short: the box is clipped by the tensor's bounds and
-            // the rows beyond arrive as zeros, still counted in the bytes
-            mbar_expect_tx(smem_u32(&bar[stg ^ 1]), kSrvTileBytes);
-            tma_load_2d(smem_u32(stage[stg ^ 1]), &map_full, 0, (int)(row0 + kSrvTileRows), smem_u32(&bar[stg ^ 1]));
-        }
         float2 s_next[2];
-        if (have_next) load_tile_scales<RANGE>(a, row0 + kSrvTileRows, lane, s_next);
+        if (have_next) load_tile_scales<RANGE>(a, row0 + kSrvTileRows, lane, wide, s_next);
 
         // Sum of the W de-quantized rows, in worker order.  Lanes past the end of the gradient
         // (only in the very last tile) decode whatever their slot of the stage holds; they are
         // never stored.
         const uint32_t row = min(row0 + lane, last_row);
         const uint32_t lb = bucket_of_row(a, row) - bucket_of_row(a, row0);
+        const float4* my_table = table + lb;
         float2 v2[16];
         bool ok = true;
         if constexpr (MODE == 2) {
             // the sum continues from the accumulator: its tile is needed before the first worker
-            ok = mbar_try_wait(smem_u32(&bar[stg]), parity);
-            if (!ok) ok = mbar_wait(smem_u32(&bar[stg]), parity);
+            ok = mbar_try_wait(bar, parity);
+            if (!ok) ok = mbar_wait(bar, parity, a.poll_limit);
             if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
-            const float4* tl = reinterpret_cast<const float4*>(stage[stg]);
+            const float4* tl = reinterpret_cast<const float4*>(stage);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float4 p = tl[swz((int)lane, c)];
@@ -263,43 +295,69 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
 
 #pragma unroll 1
         for (uint32_t g = 0; g < groups; ++g, ++u) {
-            const uint32_t cs = u % kCodeDepth, cpar = (u / kCodeDepth) & 1;
-            uint32_t* cstage = &sm.code[wid][cs][0][0];
-            bool cok = mbar_try_wait(smem_u32(&cbar[cs]), cpar);
-            if (!cok) cok = mbar_wait(smem_u32(&cbar[cs]), cpar);
-            if (!__all_sync(0xFFFFFFFFu, cok)) { failed = true; break; }
+            const uint32_t cs = u % kCodeDepth;
+            const uint32_t cstage_addr = code_base + cs * kCodeStageBytes;
+            const uint32_t* cstage = &sm.code[wid][cs][0][0] + lane * BITS;
+            cp_async_wait_group<kCodeDepth - 1>();     // this lane's pieces of the stage have landed
+            __syncwarp();                              // ... and so have the other lanes'
             const int g0 = (int)g * kGroup;
             auto decode_worker = [&](int i) {
                 uint32_t w[BITS];
-                read_stage_words<BITS>(cstage + i * (kSrvTileRows * BITS) + lane * BITS, w);
-                const float2 e = sm.table[wid][stg][((uint32_t)(g0 + i) << a.nbt_shift) + lb];
+                read_stage_words<BITS>(cstage + i * kWorkerWords, w);
+                const float4 e = my_table[(uint32_t)(g0 + i) << a.nbt_shift];
                 DecodeScale2 d;
-                d.two_h = make_float2(e.x, e.x); d.minus_h = make_float2(e.y, e.y);
+                d.two_h = make_float2(e.x, e.y); d.minus_h = make_float2(e.z, e.w);
                 add_decoded_row<BITS, RANGE>(w, d, v2, a.bias_bits);
+            };
+            // MODE 1: the parameter stage held tile k-1, whose store was committed at the end of the last
+            // iteration: once that store has read its source the stage takes tile k, which is not
+            // needed before the last worker is summed.  The load starts when half of eight workers are
+            // summed, by when the store has long read the stage.  The gradient's last tile may be short: the
+            // box is clipped by the tensor's bounds and the rows beyond arrive as zeros, still counted
+            // in the bytes.
+            auto load_params = [&]() {
+                if (lane == 0) {
+                    bulk_wait_read<0>();
+                    mbar_expect_tx(bar, kSrvTileBytes);
+                    tma_load_2d(smem_u32(stage), &map_full, 0, (int)row0, bar);
+                }
             };
             if (g0 + kGroup <= a.W) {              // a whole stage: straight-line code
 #pragma unroll
-                for (int i = 0; i < kGroup; ++i) decode_worker(i);
+                for (int i = 0; i < kGroup; ++i) {
+                    // (the two positions a whole stage can hold issue_at at: W >= 5, and W == group size)
+                    if (MODE == 1 && (i == kIssueAt % kGroup || i == kGroup - 1) && g0 + i == issue_at) load_params();
+                    decode_worker(i);
+                }
             } else {
 #pragma unroll 1
-                for (int i = 0; g0 + i < a.W; ++i) decode_worker(i);
+                for (int i = 0; g0 + i < a.W; ++i) {
+                    if (MODE == 1 && g0 + i == issue_at) load_params();
+                    decode_worker(i);
+                }
             }
             __syncwarp();                          // every lane has read the stage: refill it
             if (u + kCodeDepth < nunits)
-                fill_code_stage<BITS>(a, cstage, smem_u32(&cbar[cs]), r_begin + fill_tile * kSrvTileRows,
-                                      (int)fill_group * kGroup, lane);
+                fill_code_stage<BITS>(a, cstage_addr, r_begin + fill_tile * kSrvTileRows,
+                                      (int)fill_group * kGroup, lane_off);
+            cp_async_commit();
             if (++fill_group == groups) { fill_group = 0; ++fill_tile; }
         }
-        if (failed) break;
 
         if constexpr (MODE == 1) {
-            ok = mbar_try_wait(smem_u32(&bar[stg]), parity);
-            if (!ok) ok = mbar_wait(smem_u32(&bar[stg]), parity);
+            ok = mbar_try_wait(bar, parity);
+            if (!ok) ok = mbar_wait(bar, parity, a.poll_limit);
             if (!__all_sync(0xFFFFFFFFu, ok)) { failed = true; break; }
+        }
+        if constexpr (MODE == 0) {
+            // nothing is loaded: the stage is only written by this warp, once the store of the tile
+            // before has read it
+            if (lane == 0) bulk_wait_read<0>();
+            __syncwarp();
         }
 
         {
-            float4* tl = reinterpret_cast<float4*>(stage[stg]);
+            float4* tl = reinterpret_cast<float4*>(stage);
             const float2 nlr = make_float2(a.neg_lr, a.neg_lr);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -315,28 +373,29 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         }
         fence_proxy_async();                                   // the bulk store must see these writes
         if (have_next) {
-            // constants of the next tile; table[stg ^ 1] was last read in the previous iteration
-            store_tile_scales<BITS, RANGE>(a, sm.table[wid][stg ^ 1], lane, s_next);
+            // constants of the next tile; the table was last read before the group loop's last
+            // __syncwarp
+            store_tile_scales<BITS, RANGE>(a, table, lane, wide, s_next);
         }
         __syncwarp();
         if (lane == 0) {
             // a short last tile is clipped by the tensor's bounds
-            tma_store_2d(&map_full, 0, (int)row0, smem_u32(stage[stg]));
+            tma_store_2d(&map_full, 0, (int)row0, smem_u32(stage));
             bulk_commit();
+            if (MODE == 2 && have_next) {
+                bulk_wait_read<0>();
+                mbar_expect_tx(bar, kSrvTileBytes);
+                tma_load_2d(smem_u32(stage), &map_full, 0, (int)(row0 + kSrvTileRows), bar);
+            }
         }
     }
+    cp_async_wait_group<0>();                                  // no code copy outlives the warp
     if (lane == 0) {
         if (failed) {
+            // The tile's copy did not land within the poll limit: count it and give it one more
+            // bounded chance before the shared memory can be handed to another CTA.
             atomicAdd(timeouts, 1u);
-            // Copies that may still be in flight get a last bounded chance to land before the
-            // shared memory can be handed to another CTA: the parameter tile in use and the one
-            // issued at the top of this iteration, and the code stages issued but not consumed.
-            if (MODE != 0) {
-                mbar_wait(smem_u32(&bar[k & 1]), (k >> 1) & 1);
-                if (k + 1 < ntiles) mbar_wait(smem_u32(&bar[(k + 1) & 1]), ((k + 1) >> 1) & 1);
-            }
-            for (uint32_t j = u; j < u + kCodeDepth && j < nunits; ++j)
-                mbar_wait(smem_u32(&cbar[j % kCodeDepth]), (j / kCodeDepth) & 1);
+            mbar_wait(bar, k & 1, a.poll_limit);
         }
         bulk_wait_all<0>();                                    // stores done before the stage goes away
     }
@@ -403,10 +462,13 @@ static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, 
     CUtensorMap map_full;
     const char* why = nullptr;
     if (!encode_rows_map(&map_full, params, a.nrows_full, 4, 32, kSrvTileRows, &why)) return cudaErrorNotSupported;
-    // An ordinary launch: started as a programmatic dependent of the kernel before it, so that its
-    // CTAs become resident while that kernel drains, this kernel measured 9 us slower per launch
-    // (67 us against 58 us, eight launches back to back) - unlike the quantize kernels, which gain.
-    return launch_with_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, map_full, a, timeouts);
+    // Launched as a programmatic dependent of the kernel before it, WITHOUT releasing its own dependents
+    // early: the launch is set up while that kernel still runs and starts the moment its last CTA has
+    // gone (2.2 us per launch at every bit width, eight launches back to back).  Releasing the
+    // dependents at the top of the kernel, as the quantize kernels do, loses that again: the next
+    // launch's CTAs then take the SMs in the order in which this launch's CTAs retire, and the even
+    // split of the tiles over the SMs is gone.
+    return launch_pdl_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, map_full, a, timeouts);
 }
 
 template <int BITS, bool RANGE>
@@ -474,6 +536,7 @@ static cudaError_t launch_server_tma_codec(const WorkerPtrs& ptrs, int W, int bi
     a.W = W;
     a.neg_lr = -lr;
     a.bias_bits = 0x4B000000u;
+    a.poll_limit = kMaxWaitPolls;
     unsigned int* timeouts = wait_timeout_counter();
     if (timeouts == nullptr) return cudaErrorNotSupported;
     switch (bits) {
