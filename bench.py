@@ -16,8 +16,9 @@ Prints ONE JSON line (rank 0).  `value` is GB/s of fp32 gradient through the who
 metric with the gradients starting in pinned host memory and the updated parameters read
 back, copies inside the timed region; `roofline` describes the dominant kernel (the quantize
 kernel) and `roofline_server` the fused server kernel, both from events at the phase boundaries
-inside the timed region; `per_bits` lists both kernels for every bit width from a second,
-instrumented pass with events around every launch group; `cpu_baseline` is the scalar CPU
+inside the timed region; `per_bits` lists both kernels for every bit width, each timed on its own
+after the timed region (groups of 8 launches back to back on rotating buffers: median and best
+group; and 20 launches each between its own events); `cpu_baseline` is the scalar CPU
 checker timed on a bounded sample of the same workload.
 
 --impl reference times the CPU checker alone (rank 0 only).
@@ -318,33 +319,19 @@ def run_ours(args):
         check(lib.mqg_server_step(code_tab[b], scale_tab[b], W, b, n, B, params[b].data_ptr(), LR,
                                   None, sptr))
 
-    def step(step_no, phases=None, events=None):
+    def step(step_no, phases=None):
         """One pass of the whole path.  `phases`: three events per step (start, quantize phase done,
-        server phase done).  `events`: one pair per launch group instead (the instrumented pass
-        after the timed region; an event between two launches keeps the second from starting
-        while the first drains, so those times are a little longer than in the timed region)."""
+        server phase done); launches inside a phase run back to back."""
         if phases is not None:
             p0 = torch.cuda.Event(enable_timing=True)
             p0.record(stream)
         for b in ALL_BITS:
-            if events is not None:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
             quantize_all(b, step_no)
-            if events is not None:
-                e1.record(stream)
-                events.append(("q", b, e0, e1))
         if phases is not None:
             p1 = torch.cuda.Event(enable_timing=True)
             p1.record(stream)
         for b in ALL_BITS:
-            if events is not None:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
             server(b)
-            if events is not None:
-                e1.record(stream)
-                events.append(("s", b, e0, e1))
         if phases is not None:
             p2 = torch.cuda.Event(enable_timing=True)
             p2.record(stream)
@@ -396,10 +383,60 @@ def run_ours(args):
     q_phase_s = float(np.mean([p0.elapsed_time(p1) for p0, p1, _ in phases])) * 1e-3
     s_phase_s = float(np.mean([p1.elapsed_time(p2) for _, p1, p2 in phases])) * 1e-3
 
-    # ---- per bit width: the same steps again with events around every launch group
-    events = []
-    for i in range(args.steps):
-        step(args.warmup + args.steps + i, events=events)
+    # ---- per bit width: each kernel timed on its own, K by K.  A group is GROUP launches of the same
+    # kernel back to back between one pair of events (as they run inside a step: no event between two
+    # launches), on rotating buffer sets so that no launch finds its inputs in L2; `us` is the median
+    # over REPS groups of the group's time per launch, `us_best` the best group.  `single` figures are
+    # SINGLES launches each between its own pair of events (an event after every launch keeps the next
+    # one from being set up while it runs, so these are a few microseconds longer).
+    GROUP, REPS, SINGLES = 8, 5, 20
+
+    def time_groups(launch):
+        for i in range(2):
+            launch(i)
+        out, i = [], 2
+        for _ in range(REPS):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(GROUP):
+                launch(i)
+                i += 1
+            e1.record(stream)
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1) / GROUP)
+        return out
+
+    def time_singles(launch):
+        pairs = []
+        for i in range(SINGLES):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            launch(i)
+            e1.record(stream)
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        return [e0.elapsed_time(e1) for e0, e1 in pairs]
+
+    q_ms, s_ms, q_single, s_single = {}, {}, {}, {}
+    for b in ALL_BITS:
+        q_ms[b] = time_groups(lambda i: quantize_all(b, i))
+        q_single[b] = time_singles(lambda i: quantize_all(b, 100 + i))
+        # three sets of this width's code buffers, every parameter replica in turn: 2 launches
+        # (> 450 MB of traffic) lie between two uses of a code set, 7 between two uses of a replica
+        sets = [code_tab[b]]
+        keep = []
+        for _ in range(2):
+            cp = [t.clone() for t in codes[b]]
+            keep.append(cp)
+            sets.append((C.c_void_p * W)(*[t.data_ptr() for t in cp]))
+
+        def server_rot(i):
+            check(lib.mqg_server_step(sets[i % 3], scale_tab[b], W, b, n, B,
+                                      params[ALL_BITS[i % len(ALL_BITS)]].data_ptr(), LR, None, sptr))
+
+        s_ms[b] = time_groups(server_rot)
+        s_single[b] = time_singles(server_rot)
+        del keep, sets
     torch.cuda.synchronize()
 
     # the other way of launching the quantize phase, timed on its own for comparison
@@ -420,17 +457,13 @@ def run_ours(args):
             quantize_all(b, args.warmup + args.steps - 1)
         torch.cuda.synchronize()
 
-    q_ms = {b: [] for b in ALL_BITS}
-    s_ms = {b: [] for b in ALL_BITS}
-    for kind, b, e0, e1 in events:
-        (q_ms if kind == "q" else s_ms)[b].append(e0.elapsed_time(e1))
     peak, peak_kind = measured_hbm_peak()
     per_bits = []
     q_bytes_total = q_time_total = 0.0
     s_bytes_total = s_time_total = 0.0
     for b in ALL_BITS:
-        tq = float(np.mean(q_ms[b])) / W * 1e-3            # per worker's gradient
-        ts = float(np.mean(s_ms[b])) * 1e-3
+        tq = float(np.median(q_ms[b])) / W * 1e-3          # per worker's gradient
+        ts = float(np.median(s_ms[b])) * 1e-3
         qb, sb = quantize_bytes(n, b, B), server_bytes(n, b, B, W)
         q_bytes_total += qb * W; q_time_total += tq * W
         s_bytes_total += sb; s_time_total += ts
@@ -440,6 +473,12 @@ def run_ours(args):
             "quantize_frac_of_measured": qb / tq / 1e9 / peak, "quantize_frac_of_8tbs": qb / tq / 1e9 / NOMINAL_HBM_GBS,
             "server_us": ts * 1e6, "server_grad_gbs": 4 * n * W / ts / 1e9, "server_moved_gbs": sb / ts / 1e9,
             "server_frac_of_measured": sb / ts / 1e9 / peak, "server_frac_of_8tbs": sb / ts / 1e9 / NOMINAL_HBM_GBS,
+            "quantize_us_best": min(q_ms[b]) / W * 1e3,
+            "quantize_us_single_median": float(np.median(q_single[b])) / W * 1e3,
+            "quantize_us_single_best": min(q_single[b]) / W * 1e3,
+            "server_us_best": min(s_ms[b]) * 1e3,
+            "server_us_single_median": float(np.median(s_single[b])) * 1e3,
+            "server_us_single_best": min(s_single[b]) * 1e3,
             "wire_bytes_per_worker": mqg.mqg_wire_bytes(n, b, B),
             ("quantize_us_per_worker_launches" if batched else "quantize_us_one_launch"): other_ms[b] / W * 1e3,
         })

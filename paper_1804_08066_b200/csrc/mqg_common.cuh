@@ -60,6 +60,70 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     y[0] = c0; y[1] = c1; y[2] = c2; y[3] = c3;
 }
 
+// The part of a Philox block that is the same for every block of a launch whose counter words c1
+// (high half of the block index), c2 (worker) and the key do not change: in round 1 the product of
+// c2 and with it the new c0 and c1, in round 2 the product of that c0.  Computed once on the host
+// (philox_head), so a block costs two multiplications and one xor less.
+struct PhiloxHead {
+    uint32_t c1_r1;      // c1 after round 1: lo(M1 * worker)
+    uint32_t c0_r1;      // c0 after round 1: hi(M1 * worker) ^ c1 ^ k0[0]
+    uint32_t p0hi_r2;    // hi(M0 * c0_r1)
+    uint32_t p0lo_r2;    // lo(M0 * c0_r1) = c3 after round 2
+};
+
+__host__ __device__ inline PhiloxHead philox_head(uint32_t blk_hi, uint32_t worker, uint32_t key0)
+{
+    PhiloxHead h;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * worker;
+    h.c1_r1 = (uint32_t)p1;
+    h.c0_r1 = (uint32_t)(p1 >> 32) ^ blk_hi ^ key0;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * h.c0_r1;
+    h.p0hi_r2 = (uint32_t)(p0 >> 32);
+    h.p0lo_r2 = (uint32_t)p0;
+    return h;
+}
+
+// philox4x32_10(c0, blk_hi, worker, step) with the launch-wide part taken from `hd`.
+__device__ __forceinline__ void philox4x32_10_head(uint32_t c0, const PhiloxHead& hd, const RoundKeys& rk,
+                                                   uint32_t (&y)[4])
+{
+    // round 1: only the product of c0 depends on the block
+    const uint64_t q0 = (uint64_t)0xD2511F53u * c0;
+    uint32_t c2 = (uint32_t)(q0 >> 32) ^ rk.step ^ rk.k1[0];
+    uint32_t c3 = (uint32_t)q0;
+    // round 2: the product of c0 (= hd.c0_r1) is known
+    const uint64_t q1 = (uint64_t)0xCD9E8D57u * c2;
+    c0 = (uint32_t)(q1 >> 32) ^ hd.c1_r1 ^ rk.k0[1];
+    c2 = hd.p0hi_r2 ^ c3 ^ rk.k1[1];
+    uint32_t c1 = (uint32_t)q1;
+    c3 = hd.p0lo_r2;
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k1[r];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    y[0] = c0; y[1] = c1; y[2] = c2; y[3] = c3;
+}
+
+// The draws of a row whose four blocks are blk_lo .. blk_lo + 3 without a carry into the high half.
+__device__ __forceinline__ void draw_row_blocks_head(uint32_t blk_lo, const PhiloxHead& hd, const RoundKeys& rk,
+                                                     uint32_t (&h)[16])
+{
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        uint32_t y[4];
+        philox4x32_10_head(blk_lo + b, hd, rk, y);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) h[4 * b + k] = y[k];
+    }
+}
+
 // The 16-bit draws of the 32 elements at flat positions g0 .. g0+31, g0 % 8 == 0:
 // four Philox blocks, block index g >> 3; element g takes half (g & 1) of word (g & 7) >> 1.
 // h[j] holds the two draws of elements 2j (low half) and 2j+1 (high half).

@@ -182,7 +182,9 @@ struct TmaQuantizeShared {
 struct TmaQuantizeConsts {
     RoundKeys rk;
     uint32_t full_tiles;         // leading tiles whose rows are all complete and in range
-    uint32_t blk0_lo, blk0_hi;   // Philox block index of element 0: elem_offset / 8
+    uint32_t blk0_lo, blk0_hi;   // Philox block index of element 0: elem_offset / 8; the launch's blocks
+                                 // all have the high half blk0_hi (tma_path_applies)
+    PhiloxHead head;             // launch-wide part of the blocks of worker rk.worker
 };
 
 // What a tile needs to know about the worker it belongs to.  The one-worker kernel builds it
@@ -193,7 +195,7 @@ struct WorkerView {
     const void* grad;
     uint32_t* codes;
     float* scales;
-    uint32_t worker;             // third counter word of the draws
+    PhiloxHead head;             // launch-wide part of this worker's Philox blocks
 };
 
 // One tile, the k-th of this CTA, tile `tile` of worker `wv`.  FULL: every thread owns a complete
@@ -208,7 +210,7 @@ template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, bool NORM =
           typename Refill>
 __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
                                               const QuantizeArgs& a, const TmaQuantizeConsts& c,
-                                              uint32_t k, uint32_t tile, Refill&& refill,
+                                              uint32_t k, uint32_t rot, uint32_t tile, Refill&& refill,
                                               uint32_t local_bucket, bool scale_writer)
 {
     constexpr int kQuantStages = TmaQuantizeShared<DTYPE, THREADS>::kStages;
@@ -224,15 +226,16 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
 
     float x[32];
     if (active) {
-        if (!FULL && row >= (uint32_t)a.nrows_full)
-            stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
+        const bool ragged = !FULL && row >= (uint32_t)a.nrows_full;
+        if (ragged) stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
         read_row_swizzled<DTYPE>(stage, (int)t, x);
+        if (ragged) fence_proxy_async();     // orders those stores before the bulk copy that refills the stage
     } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j) x[j] = 0.0f;
     }
     uint32_t m;
-    uint32_t* slot = sh.slots[k % 3];
+    uint32_t* slot = sh.slots[rot];          // rot = k % 3
     if constexpr (GIVEN) {
         m = 0u;
     } else if constexpr (NORM) {
@@ -268,7 +271,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
             m = __float_as_uint(__fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3])));
         } else {
             m = slot[local_bucket];
-            if (t < THREADS / 32) sh.slots[(k + 2) % 3][t] = 0u; // next used by this CTA's tile k + 2
+            if (t < THREADS / 32) sh.slots[rot == 0 ? 2 : rot - 1][t] = 0u; // next used by this CTA's tile k + 2
         }
     }
     if (!active) return true;
@@ -289,12 +292,8 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
 
     const EncodeScale es = encode_scale<BITS>(sc);
     uint32_t h[16];
-    {
-        // Philox block of the row's first element: elem_offset / 8 + 4 * row (64-bit)
-        const uint32_t lo = c.blk0_lo + 4u * row;
-        const uint32_t hi = c.blk0_hi + (row >> 30) + (lo < c.blk0_lo ? 1u : 0u);
-        draw_row_blocks(lo, hi, wv.worker, c.rk, h);
-    }
+    // Philox blocks of the row: elem_offset / 8 + 4 * row + 0 .. 3, all in the launch's high half
+    draw_row_blocks_head(c.blk0_lo + 4u * row, wv.head, c.rk, h);
     uint32_t w[BITS];
     encode_pack_row<BITS>(x, es, h, w);
     const uint64_t word0 = (uint64_t)row * BITS;
@@ -316,7 +315,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
 // ordered bits; the kernel initialises them to the identities.
 template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, typename Refill>
 __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
-                                                    const QuantizeArgs& a, uint32_t k, uint32_t tile,
+                                                    const QuantizeArgs& a, uint32_t k, uint32_t rot, uint32_t tile,
                                                     Refill&& refill, uint32_t local_bucket, bool scale_writer)
 {
     constexpr int kQuantStages = TmaQuantizeShared<DTYPE, THREADS>::kStages;
@@ -333,9 +332,10 @@ __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THR
     float x[32];
     uint32_t mlo = kOrderedMinIdentity, mhi = kOrderedMaxIdentity;
     if (active) {
-        if (!FULL && row >= (uint32_t)a.nrows_full)
-            stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
+        const bool ragged = !FULL && row >= (uint32_t)a.nrows_full;
+        if (ragged) stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
         read_row_swizzled<DTYPE>(stage, (int)t, x);
+        if (ragged) fence_proxy_async();     // orders those stores before the bulk copy that refills the stage
         if (!FULL) {
             const uint64_t left = a.n - (uint64_t)row * 32;      // >= 1
 #pragma unroll
@@ -345,8 +345,8 @@ __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THR
         row_min_max(x, lo, hi);
         mlo = ordered_bits(lo); mhi = ordered_bits(hi);
     }
-    uint32_t* slot_hi = sh.slots[k % 3];
-    uint32_t* slot_lo = sh.slots_lo[k % 3];
+    uint32_t* slot_hi = sh.slots[rot];       // rot = k % 3
+    uint32_t* slot_lo = sh.slots_lo[rot];
     if (SHUFFLE) {
         for (uint32_t d = a.rows_per_bucket >> 1; d > 0; d >>= 1) {
             mlo = min(mlo, __shfl_xor_sync(0xFFFFFFFFu, mlo, d));
@@ -362,8 +362,8 @@ __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THR
     if (!SHUFFLE) {
         mlo = slot_lo[local_bucket]; mhi = slot_hi[local_bucket];
         if (t < THREADS / 32) {                                  // next used by this CTA's tile k + 2
-            sh.slots[(k + 2) % 3][t] = kOrderedMaxIdentity;
-            sh.slots_lo[(k + 2) % 3][t] = kOrderedMinIdentity;
+            sh.slots[rot == 0 ? 2 : rot - 1][t] = kOrderedMaxIdentity;
+            sh.slots_lo[rot == 0 ? 2 : rot - 1][t] = kOrderedMinIdentity;
         }
     }
     if (!active) return true;
@@ -428,12 +428,12 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const bool scale_writer = (t % a.rows_per_bucket) == 0;
     const uint32_t ahead = kQuantStages * stride;       // distance to the tile that refills a stage
-    const WorkerView wv = {&tmap, a.grad, a.codes, a.scales, c.rk.worker};
+    const WorkerView wv = {&tmap, a.grad, a.codes, a.scales, c.head};
 
-    uint32_t k = 0;
+    uint32_t k = 0, rot = 0;
     bool ok = true;
 #pragma unroll 1
-    for (; ok && tile < a.ntiles; tile += stride, ++k) {
+    for (; ok && tile < a.ntiles; tile += stride, ++k, rot = (rot == 2 ? 0 : rot + 1)) {
         auto refill = [&](uint32_t stage, uint32_t bar) {
             const uint32_t next_tile = tile + ahead;
             if (next_tile < a.ntiles) {
@@ -443,18 +443,18 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
         };
         if constexpr (MODE == kRange) {
             if (tile < c.full_tiles)
-                ok = range_quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, k, tile, refill,
+                ok = range_quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, k, rot, tile, refill,
                                                                                local_bucket, scale_writer);
             else
-                ok = range_quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, k, tile, refill,
+                ok = range_quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, k, rot, tile, refill,
                                                                                 local_bucket, scale_writer);
         } else {
             constexpr bool NORM = MODE == kNorm, GIVEN = MODE == kGiven;
             if (tile < c.full_tiles)
-                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM, GIVEN>(sh, wv, a, c, k, tile, refill,
+                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM, GIVEN>(sh, wv, a, c, k, rot, tile, refill,
                                                                                       local_bucket, scale_writer);
             else
-                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM, GIVEN>(sh, wv, a, c, k, tile, refill,
+                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM, GIVEN>(sh, wv, a, c, k, rot, tile, refill,
                                                                                        local_bucket, scale_writer);
         }
     }
@@ -486,6 +486,7 @@ struct WorkerTable {
     const void* grad[kMaxWorkers];
     uint32_t* codes[kMaxWorkers];
     float* scales[kMaxWorkers];
+    PhiloxHead head[kMaxWorkers];
 };
 
 template <int BITS, int DTYPE, bool SHUFFLE>
@@ -511,34 +512,48 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
     __syncthreads();
     grid_dependency_wait();            // nothing above touches global memory
 
-    auto load_tile = [&](uint32_t v, uint32_t stage, uint32_t bar) {     // thread 0 only
-        if (v < total_tiles) {
-            const uint32_t w = v / a.ntiles;
-            mbar_expect_tx(bar, box_bytes);
-            tma_load_2d(stage, &tab.map[w], 0, (int)((v - w * a.ntiles) * a.tile_rows), bar);
-        }
+    // Position in the sequence of all workers' tiles, as (worker, tile of the worker), advanced by
+    // `stride` tiles at a time without a division.
+    struct Pos { uint32_t w, tile; };
+    auto advance = [&](Pos& p, uint32_t by) {
+        p.tile += by;
+        while (p.tile >= a.ntiles) { p.tile -= a.ntiles; ++p.w; }
+    };
+    auto load_tile = [&](const Pos& p, uint32_t stage, uint32_t bar) {     // thread 0 only
+        mbar_expect_tx(bar, box_bytes);
+        tma_load_2d(stage, &tab.map[p.w], 0, (int)(p.tile * a.tile_rows), bar);
     };
     uint32_t v = blockIdx.x;
-    if (t == 0)
-        for (uint32_t s = 0; s < (uint32_t)kQuantStages; ++s)
-            load_tile(v + s * stride, smem_u32(sh.stage[s]), smem_u32(&sh.bar[s]));
+    Pos cur = {0u, 0u}, fill = {0u, 0u};   // the tile in work and the one kQuantStages turns ahead of it
+    advance(cur, v);
+    advance(fill, v);
+    uint32_t vfill = v;
+    for (uint32_t s = 0; s < (uint32_t)kQuantStages; ++s) {
+        if (t == 0 && vfill < total_tiles) load_tile(fill, smem_u32(sh.stage[s]), smem_u32(&sh.bar[s]));
+        vfill += stride;
+        if (vfill < total_tiles) advance(fill, stride);
+    }
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const bool scale_writer = (t % a.rows_per_bucket) == 0;
-    const uint32_t ahead = kQuantStages * stride;
 
-    uint32_t k = 0;
+    uint32_t k = 0, rot = 0;
     bool ok = true;
 #pragma unroll 1
-    for (; ok && v < total_tiles; v += stride, ++k) {
-        const uint32_t w = v / a.ntiles, tile = v - w * a.ntiles;
-        const WorkerView wv = {&tab.map[w], tab.grad[w], tab.codes[w], tab.scales[w], c.rk.worker + w};
-        auto refill = [&](uint32_t stage, uint32_t bar) { load_tile(v + ahead, stage, bar); };
+    for (; ok && v < total_tiles; v += stride, ++k, rot = (rot == 2 ? 0 : rot + 1)) {
+        const uint32_t w = cur.w, tile = cur.tile;
+        const WorkerView wv = {&tab.map[w], tab.grad[w], tab.codes[w], tab.scales[w], tab.head[w]};
+        auto refill = [&](uint32_t stage, uint32_t bar) {
+            if (vfill < total_tiles) load_tile(fill, stage, bar);
+        };
         if (tile < c.full_tiles)
-            ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+            ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, rot, tile, refill,
                                                                      local_bucket, scale_writer);
         else
-            ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, tile, refill,
+            ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, rot, tile, refill,
                                                                       local_bucket, scale_writer);
+        if (v + stride < total_tiles) advance(cur, stride);
+        vfill += stride;
+        if (vfill < total_tiles) advance(fill, stride);
     }
     if (!ok) {                         // as in the one-worker kernel
         if (t == 0) {
@@ -605,12 +620,23 @@ static cudaError_t launch_tma_bits(const CUtensorMap& map, const QuantizeArgs& a
 #undef MQG_TMA_CASE
 }
 
+// The Philox blocks of the launch (four per row, from block elem_offset / 8 on) all have the same
+// high half of the 64-bit block index, so that the part of a block that depends on it is a launch
+// constant (PhiloxHead) and a row's block numbers need no carry.  Fails only for a gradient that
+// straddles a multiple of 2^35 elements of the flat model; that one takes the general kernels.
+static bool blocks_share_high_half(uint64_t n, uint64_t elem_offset)
+{
+    const uint64_t first = elem_offset >> 3, last = first + 4 * ((n + 31) / 32) - 1;
+    return (first >> 32) == (last >> 32);
+}
+
 // TMA path: whole rows exist, draws are block-aligned, and a bucket is either an aligned
 // power-of-two group of at most 32 rows or a whole number of warps.
 static bool tma_path_applies(uint64_t n, uint64_t rpb, uint64_t elem_offset)
 {
     if (n < 32 * 64 || (elem_offset & 7u) != 0 || rpb == 0 || rpb > (uint64_t)kMaxTileRows) return false;
     if (n / 32 > 0x7FFFFFFFull) return false;
+    if (!blocks_share_high_half(n, elem_offset)) return false;
     return ((rpb & (rpb - 1)) == 0 && rpb <= 32) || rpb % 32 == 0;
 }
 
@@ -654,6 +680,7 @@ static int fill_tma_args(QuantizeArgs& a, TmaQuantizeConsts& c, uint64_t rpb)
     c.rk.worker = a.key.worker; c.rk.step = a.key.step;
     c.full_tiles = a.tile_rows == (uint32_t)threads ? (uint32_t)(a.nrows_full / a.tile_rows) : 0u;
     c.blk0_lo = (uint32_t)(a.elem_offset >> 3); c.blk0_hi = (uint32_t)(a.elem_offset >> 35);
+    c.head = philox_head(c.blk0_hi, c.rk.worker, c.rk.k0[0]);
     return threads;
 }
 
@@ -774,6 +801,7 @@ cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n,
         if (!encode_rows_map(&tab.map[w], grads[w], a.nrows_full, dtype == 0 ? 4 : 2, 32, a.tile_rows, &why))
             return cudaErrorNotSupported;
         tab.grad[w] = grads[w]; tab.codes[w] = codes[w]; tab.scales[w] = scales[w];
+        tab.head[w] = philox_head(c.blk0_hi, first_worker + (uint32_t)w, c.rk.k0[0]);
     }
     const uint32_t total_tiles = a.ntiles * (uint32_t)W;
     const bool shuffle = rpb <= 32;
@@ -889,6 +917,7 @@ cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, u
 bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset)
 {
     return n >= (1ull << 20) && n / 32 <= 0x7FFFFFFFull && (elem_offset & 7u) == 0 &&
+           blocks_share_high_half(n, elem_offset) &&
            (reinterpret_cast<uintptr_t>(grad) & 15u) == 0 && (reinterpret_cast<uintptr_t>(codes) & 15u) == 0;
 }
 
