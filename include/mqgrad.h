@@ -44,7 +44,8 @@ enum {
     MQG_ERR_BITS = -2,             /* bits outside 1..8 */
     MQG_ERR_ALIGN = -3,            /* a buffer is not aligned as required */
     MQG_ERR_TOO_MANY_WORKERS = -4, /* W outside 1..MQG_MAX_WORKERS */
-    MQG_ERR_CUDA = -5              /* a CUDA runtime call failed; see mqg_last_error() */
+    MQG_ERR_CUDA = -5,             /* a CUDA runtime call failed; see mqg_last_error() */
+    MQG_ERR_TIMEOUT = -6           /* a kernel's bounded wait ran out (mqg_check_timeouts) */
 };
 
 typedef enum { MQG_F32 = 0, MQG_BF16 = 1 } mqg_dtype;
@@ -297,6 +298,27 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
  * since the library was loaded in *count (0 in a healthy run).  Returns MQG_OK or MQG_ERR_CUDA.
  */
 mqg_status mqg_device_timeouts(unsigned int* count);
+
+/*
+ * The same counter as a status, for bracketing a step: synchronises with the current device, stores
+ * the number of waits that ran out since the library was loaded or since the last call with
+ * reset != 0 in *count (count may be NULL), clears the counter if reset != 0, and returns
+ * MQG_ERR_TIMEOUT when that number is not zero (the outputs of the calls enqueued on this device
+ * since the last clear are then incomplete and the step has to be repeated), else MQG_OK;
+ * MQG_ERR_CUDA if the device cannot be read.  The calls themselves are asynchronous and cannot
+ * report it: a kernel that gives up has long been enqueued with MQG_OK.  The paper has no
+ * counterpart (its transport is a blocking push / pull; Algorithm 1).
+ */
+mqg_status mqg_check_timeouts(unsigned int* count, int reset);
+
+/*
+ * TEST HOOK, process-wide, not for production use: the kernels launched after this call poll a
+ * barrier at most poll_limit times (0 restores the default), and with arm_only != 0 they arm their
+ * barriers for the bytes of a staging copy but do not issue the copy, so that the wait runs out
+ * with nothing in flight, the kernel counts it, drains and returns without writing its outputs.
+ * mqg_test_wait_override(0, 0) restores normal operation.  Always returns MQG_OK.
+ */
+mqg_status mqg_test_wait_override(uint32_t poll_limit, int arm_only);
 
 /* Message of the last error returned to the calling thread ("" if none).  Never NULL. */
 const char* mqg_last_error(void);

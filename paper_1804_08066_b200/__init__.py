@@ -10,7 +10,8 @@ Function names and argument order follow the C ABI:
   mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_quantize_minmax,
   mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_segments_l2,
   mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_quantize_1bit_ef, mqg_code_words, mqg_num_buckets,
-  mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts.
+  mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts, mqg_check_timeouts,
+  mqg_test_wait_override.
 """
 from __future__ import annotations
 
@@ -26,6 +27,7 @@ MQG_ERR_BITS = -2
 MQG_ERR_ALIGN = -3
 MQG_ERR_TOO_MANY_WORKERS = -4
 MQG_ERR_CUDA = -5
+MQG_ERR_TIMEOUT = -6
 MQG_F32, MQG_BF16 = 0, 1
 MQG_MAX_WORKERS = 32
 
@@ -50,6 +52,8 @@ def _load() -> C.CDLL:
         "mqg_last_error": (C.c_char_p, []),
         "mqg_version": (i32, []),
         "mqg_device_timeouts": (i32, [C.POINTER(C.c_uint)]),
+        "mqg_check_timeouts": (i32, [C.POINTER(C.c_uint), i32]),
+        "mqg_test_wait_override": (i32, [u32, i32]),
         "mqg_quantize": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_quantize_workers": (i32, [vp, i32, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
@@ -131,6 +135,20 @@ def mqg_device_timeouts() -> int:
     c = C.c_uint(0)
     _check(_lib.mqg_device_timeouts(C.byref(c)))
     return int(c.value)
+
+
+def mqg_check_timeouts(reset: bool = True) -> int:
+    """Waits that ran out on the current device since the last reset (synchronises).  Raises MqgError
+    with status MQG_ERR_TIMEOUT when there were any, after clearing the counter if `reset`; returns 0
+    otherwise."""
+    c = C.c_uint(0)
+    _check(_lib.mqg_check_timeouts(C.byref(c), 1 if reset else 0))
+    return int(c.value)
+
+
+def mqg_test_wait_override(poll_limit: int = 0, arm_only: bool = False) -> None:
+    """Test hook of the C ABI (see include/mqgrad.h); (0, False) restores normal operation."""
+    _check(_lib.mqg_test_wait_override(poll_limit, 1 if arm_only else 0))
 
 
 def _grad_dtype(grad) -> int:

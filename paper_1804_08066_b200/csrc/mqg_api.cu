@@ -151,6 +151,22 @@ mqg_status mqg_device_timeouts(unsigned int* count)
     return MQG_OK;
 }
 
+mqg_status mqg_check_timeouts(unsigned int* count, int reset)
+{
+    unsigned int c = 0;
+    const cudaError_t err = mqg::read_wait_timeouts(&c, reset != 0);
+    if (err != cudaSuccess) return cuda_fail("mqg_check_timeouts", err);
+    if (count) *count = c;
+    if (c != 0) return fail(MQG_ERR_TIMEOUT, "%u bounded wait(s) of a kernel ran out on this device", c);
+    return MQG_OK;
+}
+
+mqg_status mqg_test_wait_override(uint32_t poll_limit, int arm_only)
+{
+    mqg::set_wait_policy(poll_limit, arm_only != 0 ? 1u : 0u);
+    return MQG_OK;
+}
+
 mqg_status mqg_quantize(const void* grad, uint64_t n, int bits, uint64_t bucket, uint64_t seed,
                         uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
                         uint32_t step, uint64_t elem_offset, void* cuda_stream)

@@ -30,6 +30,8 @@ struct QuantizeArgs {
     uint64_t nrows_full;    // floor(n / 32): rows the tensor map covers
     uint32_t ntiles;
     DrawKey key;
+    uint32_t poll_limit;        // polls of one barrier wait before the CTA gives up (TMA kernels)
+    uint32_t arm_only;          // test hook: 1 = arm the barriers but issue no copy
 };
 
 // Max over the rows of each bucket of the tile.  `m` is this thread's row max (bit pattern of
@@ -222,7 +224,7 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     uint8_t* stage = sh.stage[stg];
 
     bool ok = mbar_try_wait(bar, parity);
-    if (!ok) ok = mbar_wait(bar, parity);
+    if (!ok) ok = mbar_wait(bar, parity, a.poll_limit);
 
     float x[32];
     if (active) {
@@ -327,7 +329,7 @@ __device__ __forceinline__ bool range_quantize_tile(TmaQuantizeShared<DTYPE, THR
     uint8_t* stage = sh.stage[stg];
 
     bool ok = mbar_try_wait(bar, parity);
-    if (!ok) ok = mbar_wait(bar, parity);
+    if (!ok) ok = mbar_wait(bar, parity, a.poll_limit);
 
     float x[32];
     uint32_t mlo = kOrderedMinIdentity, mhi = kOrderedMaxIdentity;
@@ -421,8 +423,9 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
     if (t == 0) {
         for (uint32_t s = 0; s < (uint32_t)kQuantStages && tile + s * stride < a.ntiles; ++s) {
             mbar_expect_tx(smem_u32(&sh.bar[s]), box_bytes);
-            tma_load_2d(smem_u32(sh.stage[s]), &tmap, 0, (int)((tile + s * stride) * a.tile_rows),
-                        smem_u32(&sh.bar[s]));
+            if (!a.arm_only)
+                tma_load_2d(smem_u32(sh.stage[s]), &tmap, 0, (int)((tile + s * stride) * a.tile_rows),
+                            smem_u32(&sh.bar[s]));
         }
     }
     const uint32_t local_bucket = t / a.rows_per_bucket;
@@ -438,7 +441,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
             const uint32_t next_tile = tile + ahead;
             if (next_tile < a.ntiles) {
                 mbar_expect_tx(bar, box_bytes);
-                tma_load_2d(stage, &tmap, 0, (int)(next_tile * a.tile_rows), bar);
+                if (!a.arm_only) tma_load_2d(stage, &tmap, 0, (int)(next_tile * a.tile_rows), bar);
             }
         };
         if constexpr (MODE == kRange) {
@@ -467,7 +470,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
             atomicAdd(timeouts, 1u);
             uint32_t j = k - 1, tl = tile - stride;
             for (int s = 0; s < kQuantStages && tl < a.ntiles; ++s, ++j, tl += stride)
-                mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1);
+                mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1, a.poll_limit);
         }
         __syncthreads();
     }
@@ -521,7 +524,7 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
     };
     auto load_tile = [&](const Pos& p, uint32_t stage, uint32_t bar) {     // thread 0 only
         mbar_expect_tx(bar, box_bytes);
-        tma_load_2d(stage, &tab.map[p.w], 0, (int)(p.tile * a.tile_rows), bar);
+        if (!a.arm_only) tma_load_2d(stage, &tab.map[p.w], 0, (int)(p.tile * a.tile_rows), bar);
     };
     uint32_t v = blockIdx.x;
     Pos cur = {0u, 0u}, fill = {0u, 0u};   // the tile in work and the one kQuantStages turns ahead of it
@@ -560,7 +563,7 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
             atomicAdd(timeouts, 1u);
             uint32_t j = k - 1, vl = v - stride;
             for (int s = 0; s < kQuantStages && vl < total_tiles; ++s, ++j, vl += stride)
-                mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1);
+                mbar_wait(smem_u32(&sh.bar[j % kQuantStages]), (j / kQuantStages) & 1, a.poll_limit);
         }
         __syncthreads();
     }
@@ -659,6 +662,9 @@ static uint64_t fill_args(QuantizeArgs& a, const void* grad, uint64_t n, int bit
     a.key.seed_lo = (uint32_t)seed; a.key.seed_hi = (uint32_t)(seed >> 32);
     a.key.worker = worker; a.key.step = step;
     a.nrows_full = n / 32;
+    const WaitPolicy policy = wait_policy();
+    a.poll_limit = policy.poll_limit;
+    a.arm_only = policy.arm_only;
     return rpb;
 }
 

@@ -49,6 +49,7 @@ struct ServerTmaArgs {
     float neg_lr;
     uint32_t bias_bits;          // 0x4B000000 (2^23), a run-time constant for the byte permutes
     uint32_t poll_limit;         // polls of one barrier wait before the warp gives up
+    uint32_t arm_only;           // test hook: 1 = arm the barriers but issue no parameter copy
 };
 
 // Dynamic shared memory of one CTA (base rounded up to 1024 bytes for the 128-byte swizzle).
@@ -244,7 +245,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         store_tile_scales<BITS, RANGE>(a, table, lane, wide, s0);
         if (MODE == 2 && lane == 0) {
             mbar_expect_tx(bar, kSrvTileBytes);
-            tma_load_2d(smem_u32(stage), &map_full, 0, (int)r_begin, bar);
+            if (!a.arm_only) tma_load_2d(smem_u32(stage), &map_full, 0, (int)r_begin, bar);
         }
         // the first kCodeDepth code stages (u2 = stage number, tile u2 / groups, group u2 % groups);
         // one copy group per stage, empty when there is no such stage
@@ -319,7 +320,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
                 if (lane == 0) {
                     bulk_wait_read<0>();
                     mbar_expect_tx(bar, kSrvTileBytes);
-                    tma_load_2d(smem_u32(stage), &map_full, 0, (int)row0, bar);
+                    if (!a.arm_only) tma_load_2d(smem_u32(stage), &map_full, 0, (int)row0, bar);
                 }
             };
             if (g0 + kGroup <= a.W) {              // a whole stage: straight-line code
@@ -385,7 +386,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
             if (MODE == 2 && have_next) {
                 bulk_wait_read<0>();
                 mbar_expect_tx(bar, kSrvTileBytes);
-                tma_load_2d(smem_u32(stage), &map_full, 0, (int)(row0 + kSrvTileRows), bar);
+                if (!a.arm_only) tma_load_2d(smem_u32(stage), &map_full, 0, (int)(row0 + kSrvTileRows), bar);
             }
         }
     }
@@ -536,7 +537,9 @@ static cudaError_t launch_server_tma_codec(const WorkerPtrs& ptrs, int W, int bi
     a.W = W;
     a.neg_lr = -lr;
     a.bias_bits = 0x4B000000u;
-    a.poll_limit = kMaxWaitPolls;
+    const WaitPolicy policy = wait_policy();
+    a.poll_limit = policy.poll_limit;
+    a.arm_only = policy.arm_only;
     unsigned int* timeouts = wait_timeout_counter();
     if (timeouts == nullptr) return cudaErrorNotSupported;
     switch (bits) {

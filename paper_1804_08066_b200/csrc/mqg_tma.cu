@@ -1,5 +1,6 @@
 // Host side of the TMA helpers: tensor-map encoding through the driver entry point (so the
 // library needs no link-time dependency on libcuda) and the per-device timeout counter.
+#include <atomic>
 #include <mutex>
 
 #include "mqg_tma.cuh"
@@ -72,9 +73,33 @@ unsigned int* wait_timeout_counter()
     return g_counter_ptr[dev];
 }
 
-cudaError_t read_wait_timeouts(unsigned int* count)
+cudaError_t read_wait_timeouts(unsigned int* count, bool reset)
 {
-    return cudaMemcpyFromSymbol(count, g_wait_timeouts, sizeof(unsigned int), 0, cudaMemcpyDeviceToHost);
+    cudaError_t err = cudaMemcpyFromSymbol(count, g_wait_timeouts, sizeof(unsigned int), 0, cudaMemcpyDeviceToHost);
+    if (err == cudaSuccess && reset && *count != 0) {
+        const unsigned int zero = 0;
+        err = cudaMemcpyToSymbol(g_wait_timeouts, &zero, sizeof(unsigned int), 0, cudaMemcpyHostToDevice);
+    }
+    return err;
+}
+
+namespace {
+std::atomic<uint32_t> g_poll_limit{kMaxWaitPolls};
+std::atomic<uint32_t> g_arm_only{0};
+}  // namespace
+
+WaitPolicy wait_policy()
+{
+    WaitPolicy p;
+    p.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
+    p.arm_only = g_arm_only.load(std::memory_order_relaxed);
+    return p;
+}
+
+void set_wait_policy(uint32_t poll_limit, uint32_t arm_only)
+{
+    g_poll_limit.store(poll_limit == 0 ? kMaxWaitPolls : poll_limit, std::memory_order_relaxed);
+    g_arm_only.store(arm_only ? 1u : 0u, std::memory_order_relaxed);
 }
 
 }  // namespace mqg

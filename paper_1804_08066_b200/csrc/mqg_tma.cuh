@@ -171,7 +171,18 @@ bool encode_rows_map(CUtensorMap* map, const void* base, uint64_t rows, int elem
 // library's own device image; kernels receive the pointer as an argument).  nullptr on error.
 unsigned int* wait_timeout_counter();
 
-// Reads that counter (synchronises with the device).  Returns cudaSuccess and the count.
-cudaError_t read_wait_timeouts(unsigned int* count);
+// Reads that counter (synchronises with the device) and, with `reset`, clears it.
+cudaError_t read_wait_timeouts(unsigned int* count, bool reset = false);
+
+// What the launchers put into their kernels' arguments: the poll limit of a barrier wait, and
+// whether the staging copies are issued at all.  The defaults are kMaxWaitPolls and true; the
+// test hook mqg_test_wait_override() changes them for the whole process, so that a test can make
+// a wait run out with nothing in flight.
+struct WaitPolicy {
+    uint32_t poll_limit;
+    uint32_t arm_only;       // 1: barriers are armed for their bytes but no copy is issued
+};
+WaitPolicy wait_policy();
+void set_wait_policy(uint32_t poll_limit, uint32_t arm_only);
 
 }  // namespace mqg
