@@ -650,6 +650,13 @@ def run_ours(args):
            "h2d_bytes_per_step": grad_bytes_per_step, "d2h_bytes_per_step": len(ALL_BITS) * 4 * n,
            "ms_per_step": e2e_ms, "steps": e2e_steps}
 
+    # ---- the other workloads of the specification (single-GPU run only; outside `value`)
+    other_configs = None
+    if rank == 0 and world == 1 and not args.no_configs:
+        import bench_configs
+        torch.cuda.empty_cache()
+        other_configs = bench_configs.run_all(torch, mqg, lib, check, peak)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu, _ = cpu_baseline(host_grads)
@@ -667,6 +674,8 @@ def run_ours(args):
             "variant_1bit_ef": variant_1bit_ef,
             "per_bits": per_bits,
         }
+        if other_configs is not None:
+            line["configs"] = other_configs
         if cpu is not None:
             line["cpu_baseline"] = cpu
         print(json.dumps(line))
@@ -716,6 +725,19 @@ def run_single_kernel(args):
         launch = lambda i: mqg.mqg_quantize_segments(grads[i % rot], seg, coff, b, PHILOX_SEED, codes[i % rot],
                                                      scales[i % rot], worker=i % rot, step=i)
         nbytes = 8 * n + 4 * int(coff[-1])
+    elif args.kernel == "quantize_segments_workers":
+        # the layered gradient of W workers in one call (three launches)
+        sizes = [int(np.prod(sh)) for sh in wl.ALEXNET_SHAPES]
+        n = sum(sizes)
+        seg = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+        coff = np.concatenate([[0], np.cumsum([mqg.mqg_code_words(sz, b) for sz in sizes])]).astype(np.uint64)
+        rot = 2
+        grads = [torch.from_numpy(wl.layered(sizes, config=3, worker=w)).cuda() for w in range(W)]
+        codes = [[torch.zeros(int(coff[-1]), dtype=torch.int32, device="cuda") for _ in range(W)] for _ in range(rot)]
+        scales = [[torch.zeros(len(sizes), dtype=torch.float32, device="cuda") for _ in range(W)] for _ in range(rot)]
+        launch = lambda i: mqg.mqg_quantize_segments_workers(grads, W, seg, coff, b, PHILOX_SEED, codes[i % rot],
+                                                             scales[i % rot], first_worker=0, step=i)
+        nbytes = W * (8 * n + 4 * int(coff[-1]))
     elif args.kernel == "server_segments":
         # fused server step on the layered gradient (per-layer scale), W workers
         sizes = [int(np.prod(sh)) for sh in wl.ALEXNET_SHAPES]
@@ -808,11 +830,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the other workloads of the specification (`configs` in the JSON line)")
     ap.add_argument("--quantize-launch", choices=["batched", "per-worker"], default="batched",
                     help="the step's quantize phase: one mqg_quantize_workers launch per bit width for all "
                          "workers' gradients, or one mqg_quantize launch per worker")
     ap.add_argument("--kernel", choices=["quantize", "quantize_workers", "server", "requantize", "quantize_l2", "onebit",
-                             "quantize_segments", "server_segments"],
+                             "quantize_segments", "quantize_segments_workers", "server_segments"],
                     default=None,
                     help="run a few launches of one kernel on a small case instead of the benchmark")
     ap.add_argument("--bits", type=int, default=4)

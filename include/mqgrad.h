@@ -264,7 +264,7 @@ mqg_status mqg_quantize_segments_l2_static(const void* grad, int nseg, const uin
                                            void* cuda_stream);
 
 /*
- * Per-layer scale ("gradient quantization is applied to these two layers", Section 4.1): the flat
+ * Per-layer scale (Section 4.1 quantizes the two large fully connected layers, each as a whole): the flat
  * gradient is cut into nseg segments; segment j = elements [seg_off[j], seg_off[j+1]) is ONE bucket
  * with scale scales[j], and its bit stream starts on a word boundary at word code_off[j].
  *   seg_off   [in] HOST array of nseg+1 non-decreasing element offsets (seg_off[0] may be > 0)
@@ -283,6 +283,23 @@ mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg
                                  const uint64_t* code_off, int bits, uint64_t seed,
                                  uint32_t* codes, float* scales, mqg_dtype dtype, uint32_t worker,
                                  uint32_t step, uint64_t elem_offset, void* cuda_stream);
+
+/*
+ * mqg_quantize_segments for W workers' gradients that share one segment table, in three launches for
+ * all of them (zero the scales, max pass, encode pass) instead of five per worker - the per-layer
+ * counterpart of mqg_quantize_workers, for a host that plays several workers on one device (all
+ * workers run Quantize(g, K) with the same K in an iteration; Algorithm 1, WorkerIterate line 3).
+ *   grads/codes/scales [in] HOST arrays of W device pointers; worker w draws with worker id
+ *                      first_worker + w; codes[w] takes code_off[nseg] words, scales[w] nseg floats
+ * Worker w's outputs are bit-identical to mqg_quantize_segments(grads[w], ..., first_worker + w, ...).
+ * Errors as mqg_quantize_segments, per worker; MQG_ERR_TOO_MANY_WORKERS for W outside
+ * 1..MQG_MAX_WORKERS.
+ */
+mqg_status mqg_quantize_segments_workers(const void* const* grads, int W, int nseg, const uint64_t* seg_off,
+                                         const uint64_t* code_off, int bits, uint64_t seed,
+                                         uint32_t* const* codes, float* const* scales, mqg_dtype dtype,
+                                         uint32_t first_worker, uint32_t step, uint64_t elem_offset,
+                                         void* cuda_stream);
 
 /* mqg_server_step for buffers written by mqg_quantize_segments (same segment tables). */
 mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* const* scales, int W,

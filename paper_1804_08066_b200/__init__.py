@@ -7,7 +7,7 @@ raises.
 
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
-  mqg_server_requantize, mqg_quantize_segments, mqg_server_step_segments, mqg_quantize_minmax,
+  mqg_server_requantize, mqg_quantize_segments, mqg_quantize_segments_workers, mqg_server_step_segments, mqg_quantize_minmax,
   mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_segments_l2,
   mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_quantize_1bit_ef, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts, mqg_check_timeouts,
@@ -65,6 +65,7 @@ def _load() -> C.CDLL:
         "mqg_server_requantize": (i32, [vp, vp, i32, i32, u64, u64, f32, u64, vp, vp, u32, u32, vp]),
         "mqg_quantize_segments": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_server_step_segments": (i32, [vp, vp, i32, i32, i32, vp, vp, vp, f32, vp, vp]),
+        "mqg_quantize_segments_workers": (i32, [vp, i32, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_quantize_1bit_ef": (i32, [vp, vp, u64, u64, vp, vp, i32, vp]),
         "mqg_quantize_l2": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_l2_workspace_floats": (C.c_size_t, [i32, vp]),
@@ -78,7 +79,20 @@ def _load() -> C.CDLL:
     return lib
 
 
-_lib = _load()
+class _LazyLibrary:
+    """Loads libmqgrad.so at the first call instead of at import, so that a process which only
+    imports the input generators (workloads.py) never maps the library."""
+
+    def __init__(self):
+        self._lib = None
+
+    def __getattr__(self, name):
+        if self._lib is None:
+            self._lib = _load()
+        return getattr(self._lib, name)
+
+
+_lib = _LazyLibrary()
 
 
 def _check(status: int) -> None:
@@ -245,6 +259,15 @@ def mqg_quantize_segments(grad, seg_off, code_off, bits: int, seed: int, codes, 
                                       _grad_dtype(grad), worker, step, elem_offset, _stream()))
 
 
+def mqg_quantize_segments_workers(grads, W: int, seg_off, code_off, bits: int, seed: int, codes, scales,
+                                  first_worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    nseg = len(seg_off) - 1
+    _check(_lib.mqg_quantize_segments_workers(_ptr_table(grads, "grads"), W, nseg, _u64_table(seg_off),
+                                              _u64_table(code_off), bits, seed & 0xFFFFFFFFFFFFFFFF,
+                                              _ptr_table(codes, "codes"), _ptr_table(scales, "scales"),
+                                              _grad_dtype(grads[0]), first_worker, step, elem_offset, _stream()))
+
+
 def mqg_server_step_segments(codes, scales, W: int, bits: int, seg_off, code_off, params,
                              lr: float, acc_out=None) -> None:
     nseg = len(seg_off) - 1
@@ -301,4 +324,5 @@ def mqg_quantize_segments_l2_static(grad, seg_off, code_off, bits: int, seed: in
 
 def raw_library() -> C.CDLL:
     """The ctypes handle, for callers that pass raw device pointers themselves."""
-    return _lib
+    _lib.mqg_version                       # loads the library if this is its first use
+    return _lib._lib

@@ -2,6 +2,8 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <utility>
+#include <vector>
 
 #include "../../include/mqgrad.h"
 #include "mqg_common.cuh"
@@ -408,6 +410,89 @@ mqg_status mqg_quantize_segments(const void* grad, int nseg, const uint64_t* seg
             static_cast<const char*>(grad) + seg_off[j] * esz, seg_off[j + 1] - seg_off[j], bits, seed,
             codes + code_off[j], scales + j, (int)dtype, worker, step, elem_offset + seg_off[j], stream);
         if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments", err);
+    }
+    return MQG_OK;
+}
+
+mqg_status mqg_quantize_segments_workers(const void* const* grads, int W, int nseg, const uint64_t* seg_off,
+                                         const uint64_t* code_off, int bits, uint64_t seed,
+                                         uint32_t* const* codes, float* const* scales, mqg_dtype dtype,
+                                         uint32_t first_worker, uint32_t step, uint64_t elem_offset,
+                                         void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (W < 1 || W > MQG_MAX_WORKERS)
+        return fail(MQG_ERR_TOO_MANY_WORKERS, "W = %d is outside 1..%d", W, MQG_MAX_WORKERS);
+    if (nseg < 0) return fail(MQG_ERR_INVALID, "nseg = %d is negative", nseg);
+    if (nseg == 0) return MQG_OK;
+    if (!grads || !codes || !scales) return fail(MQG_ERR_INVALID, "grads, codes or scales pointer table is null");
+    for (int w = 0; w < W; ++w) {
+        if (!grads[w] || !codes[w] || !scales[w])
+            return fail(MQG_ERR_INVALID, "worker %d: grad, codes or scales is null", w);
+        if (!aligned16(grads[w])) return fail(MQG_ERR_ALIGN, "worker %d: grad not 16-byte aligned", w);
+        if (!aligned16(codes[w])) return fail(MQG_ERR_ALIGN, "worker %d: codes not 16-byte aligned", w);
+        if (!aligned4(scales[w])) return fail(MQG_ERR_ALIGN, "worker %d: scales not 4-byte aligned", w);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t esz = dtype == MQG_BF16 ? 2 : 4;
+    // a long segment whose buffers are aligned for bulk copies with every worker is an entry of the
+    // TMA-fed part of the encode launch; all other segments go through its table-driven part
+    auto own = [&](int j) {
+        for (int w = 0; w < W; ++w)
+            if (!mqg::quantize_given_scale_applies(static_cast<const char*>(grads[w]) + seg_off[j] * esz,
+                                                   seg_off[j + 1] - seg_off[j], codes[w] + code_off[j],
+                                                   elem_offset + seg_off[j]))
+                return false;
+        return true;
+    };
+    bool zeroed = false;
+    mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            if (!zeroed) {                 // after the table has been validated
+                const cudaError_t err = mqg::launch_zero_scales(scales, W, nseg, stream);
+                if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_workers", err);
+                zeroed = true;
+            }
+            const cudaError_t err = mqg::launch_absmax_workers(grads, scales, first, W, tab, (int)dtype, stream);
+            if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_workers", err);
+            return MQG_OK;
+        });
+    if (st != MQG_OK) return st;
+
+    std::vector<mqg::SegEntryHost> entries;
+    for (int j = 0; j < nseg; ++j) {
+        if (seg_off[j + 1] == seg_off[j] || !own(j)) continue;
+        for (int w = 0; w < W; ++w) {
+            mqg::SegEntryHost e;
+            e.grad = static_cast<const char*>(grads[w]) + seg_off[j] * esz;
+            e.codes = codes[w] + code_off[j];
+            e.scale = scales[w] + j;
+            e.n = seg_off[j + 1] - seg_off[j];
+            e.elem_offset = elem_offset + seg_off[j];
+            e.worker = first_worker + (uint32_t)w;
+            entries.push_back(e);
+        }
+    }
+    std::vector<std::pair<mqg::SegmentTable, int>> short_tabs;
+    st = for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            if (tab.tile_start[tab.nseg] != 0) short_tabs.emplace_back(tab, first);
+            return MQG_OK;
+        }, own);
+    if (st != MQG_OK) return st;
+    const size_t per = (size_t)mqg::kMaxSegEntriesPerLaunch;
+    const size_t entry_launches = (entries.size() + per - 1) / per;
+    const size_t launches = entry_launches > short_tabs.size() ? entry_launches : short_tabs.size();
+    for (size_t i = 0; i < launches; ++i) {
+        const size_t e0 = i * per;
+        const int nent = e0 < entries.size() ? (int)(entries.size() - e0 < per ? entries.size() - e0 : per) : 0;
+        const mqg::SegmentTable* tab = i < short_tabs.size() ? &short_tabs[i].first : nullptr;
+        const int first = i < short_tabs.size() ? short_tabs[i].second : 0;
+        const cudaError_t err = mqg::launch_encode_workers(nent ? entries.data() + e0 : nullptr, nent, tab, grads,
+                                                           codes, scales, first, W, bits, seed, (int)dtype,
+                                                           first_worker, step, elem_offset, stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_quantize_segments_workers", err);
     }
     return MQG_OK;
 }

@@ -91,6 +91,26 @@ cudaError_t launch_quantize_given_scale(const void* grad, uint64_t n, int bits, 
                                         float* scale, int dtype, uint32_t worker, uint32_t step,
                                         uint64_t elem_offset, cudaStream_t stream);
 
+// Per-layer quantization of several workers in three launches (mqg_segments_workers.cu): zero the
+// scale arrays, max pass over all (worker, segment) pairs, one encode pass.  A SegEntryHost is one
+// (worker, long segment) pair for which quantize_given_scale_applies() holds.
+struct SegEntryHost {
+    const void* grad;        // the segment's first element
+    uint32_t* codes;         // its first code word
+    float* scale;            // its scale
+    uint64_t n;              // its length
+    uint64_t elem_offset;    // flat position of its first element (for the draws)
+    uint32_t worker;         // worker id of the draws
+};
+constexpr int kMaxSegEntriesPerLaunch = 32;
+cudaError_t launch_zero_scales(float* const* scales, int W, int nseg, cudaStream_t stream);
+cudaError_t launch_absmax_workers(const void* const* grads, float* const* scales, int first, int W,
+                                  const SegmentTable& tab, int dtype, cudaStream_t stream);
+cudaError_t launch_encode_workers(const SegEntryHost* entries, int nent, const SegmentTable* short_tab,
+                                  const void* const* grads, uint32_t* const* codes, float* const* scales,
+                                  int scale_first, int W, int bits, uint64_t seed, int dtype,
+                                  uint32_t first_worker, uint32_t step, uint64_t elem_offset, cudaStream_t stream);
+
 // Two-pass quantize with uniform large buckets (bucket > kMaxFusedBucket, or a single bucket
 // whose length is not a multiple of 32).
 cudaError_t launch_quantize_big_buckets(const void* grad, uint64_t n, int bits, uint64_t bucket,

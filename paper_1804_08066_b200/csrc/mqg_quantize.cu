@@ -9,30 +9,11 @@
 // from HBM exactly once.
 #include <string.h>
 
-#include "mqg_common.cuh"
-#include "mqg_internal.h"
-#include "mqg_tma.cuh"
+#include <atomic>
+
+#include "mqg_quantize_tile.cuh"
 
 namespace mqg {
-
-struct QuantizeArgs {
-    const void* grad;
-    uint32_t* codes;
-    float* scales;
-    uint64_t n;             // elements
-    uint64_t nrows;         // ceil(n / 32)
-    uint64_t nbuckets;      // ceil(n / bucket)
-    uint64_t ncode_words;   // ceil(n * bits / 32)
-    uint64_t elem_offset;
-    uint32_t rows_per_bucket;   // bucket / 32 (a single ragged bucket counts as "all rows")
-    uint32_t tile_rows;         // rows per tile: a multiple of rows_per_bucket, <= 256
-    uint32_t buckets_per_tile;
-    uint64_t nrows_full;    // floor(n / 32): rows the tensor map covers
-    uint32_t ntiles;
-    DrawKey key;
-    uint32_t poll_limit;        // polls of one barrier wait before the CTA gives up (TMA kernels)
-    uint32_t arm_only;          // test hook: 1 = arm the barriers but issue no copy
-};
 
 // Max over the rows of each bucket of the tile.  `m` is this thread's row max (bit pattern of
 // a non-negative float, so unsigned order = float order).  Returns the bucket's max.
@@ -120,195 +101,6 @@ quantize_pack_kernel(const QuantizeArgs a)
 }
 
 
-// ---------------------------------------------------------------------------------------
-// The same computation fed by TMA: a persistent CTA walks tiles blockIdx.x, +gridDim.x, ...;
-// one elected thread keeps STAGES tiled bulk copies (cp.async.bulk.tensor, 128- or 64-byte
-// swizzle) in flight into a shared-memory ring, each completing on its own mbarrier, so the
-// compute warps never issue a global load and never wait for DRAM latency in steady state.
-// One __syncthreads per tile publishes the bucket maxima and releases the stage for refill.
-// ---------------------------------------------------------------------------------------
-template <int DTYPE>
-__device__ __forceinline__ void read_row_swizzled(const uint8_t* stage, int row, float (&x)[32])
-{
-    if constexpr (DTYPE == 0) {
-        read_row(reinterpret_cast<const float4*>(stage), row, x);
-    } else {
-        const uint4* t = reinterpret_cast<const uint4*>(stage);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint4 v = t[row * 4 + (c ^ ((row >> 1) & 3))];
-            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                x[8 * c + 2 * k] = bf16_lo(u[k]);
-                x[8 * c + 2 * k + 1] = bf16_hi(u[k]);
-            }
-        }
-    }
-}
-
-// The one row of the gradient that is shorter than 32 elements is not covered by the tensor
-// map: its owner copies it (zero-padded) into its own row of the stage with plain loads and
-// then reads it back like any other row.
-template <int DTYPE>
-__device__ __noinline__ void stage_ragged_row(uint8_t* stage, int row, const void* grad, uint64_t e0,
-                                              uint64_t n)
-{
-    for (int j = 0; j < 32; ++j) {
-        const bool in = e0 + j < n;
-        if constexpr (DTYPE == 0) {
-            float* tf = reinterpret_cast<float*>(stage);
-            tf[swz(row, j >> 2) * 4 + (j & 3)] = in ? static_cast<const float*>(grad)[e0 + j] : 0.0f;
-        } else {
-            uint16_t* th = reinterpret_cast<uint16_t*>(stage);
-            const int chunk = (j >> 3) ^ ((row >> 1) & 3);
-            th[(row * 4 + chunk) * 8 + (j & 7)] = in ? static_cast<const uint16_t*>(grad)[e0 + j] : (uint16_t)0;
-        }
-    }
-}
-
-template <int DTYPE, int THREADS>
-struct TmaQuantizeShared {
-    static constexpr int kRowBytes = DTYPE == 0 ? 128 : 64;
-    // depth of the shared-memory ring: two stages where they fit in 32 KB, else one (the refill
-    // of a single stage still hides behind the tile's arithmetic)
-    static constexpr int kStages = 2 * THREADS * kRowBytes <= 32768 ? 2 : 1;
-    alignas(1024) uint8_t stage[kStages][THREADS * kRowBytes];
-    uint32_t slots[3][THREADS / 32];       // bucket maxima, rotating so no reset races a use
-    uint32_t slots_lo[3][THREADS / 32];    // bucket minima of the (min, max) variant, as ordered bits
-    alignas(8) uint64_t bar[kStages];
-};
-
-// Kernel-constant inputs of the TMA kernel beyond QuantizeArgs: the ten Philox round keys are
-// computed on the host so the kernel reads them as constant operands.
-struct TmaQuantizeConsts {
-    RoundKeys rk;
-    uint32_t full_tiles;         // leading tiles whose rows are all complete and in range
-    uint32_t blk0_lo, blk0_hi;   // Philox block index of element 0: elem_offset / 8; the launch's blocks
-                                 // all have the high half blk0_hi (tma_path_applies)
-    PhiloxHead head;             // launch-wide part of the blocks of worker rk.worker
-};
-
-// What a tile needs to know about the worker it belongs to.  The one-worker kernel builds it
-// from its kernel parameters (so every member stays a constant operand), the batched kernel from
-// its table.
-struct WorkerView {
-    const CUtensorMap* map;
-    const void* grad;
-    uint32_t* codes;
-    float* scales;
-    PhiloxHead head;             // launch-wide part of this worker's Philox blocks
-};
-
-// One tile, the k-th of this CTA, tile `tile` of worker `wv`.  FULL: every thread owns a complete
-// row (no bounds checks).  SHUFFLE: a bucket is an aligned power-of-two group of at most 32 rows
-// (lane shuffles); otherwise a whole number of warps (one shared-memory atomic per warp).  After
-// the tile's rows are in registers thread 0 calls `refill(stage, bar)` to start the copy that
-// uses the stage next.  Returns false if the tile's copy never landed.
-// GIVEN: the scale is not computed here: every tile belongs to one bucket whose scale already stands
-// at wv.scales[0] (per-layer quantization after its max or norm pass); no reduction, no scale written
-// except that a raw maximum below the flush limit is replaced by 0 by the first tile.
-template <int BITS, int DTYPE, int THREADS, bool FULL, bool SHUFFLE, bool NORM = false, bool GIVEN = false,
-          typename Refill>
-__device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>& sh, const WorkerView wv,
-                                              const QuantizeArgs& a, const TmaQuantizeConsts& c,
-                                              uint32_t k, uint32_t rot, uint32_t tile, Refill&& refill,
-                                              uint32_t local_bucket, bool scale_writer)
-{
-    constexpr int kQuantStages = TmaQuantizeShared<DTYPE, THREADS>::kStages;
-    const uint32_t t = threadIdx.x;
-    const uint32_t row = tile * a.tile_rows + t;
-    const bool active = FULL || (t < a.tile_rows && row < (uint32_t)a.nrows);
-    const uint32_t stg = k % kQuantStages, parity = (k / kQuantStages) & 1;
-    const uint32_t bar = smem_u32(&sh.bar[stg]);
-    uint8_t* stage = sh.stage[stg];
-
-    bool ok = mbar_try_wait(bar, parity);
-    if (!ok) ok = mbar_wait(bar, parity, a.poll_limit);
-
-    float x[32];
-    if (active) {
-        const bool ragged = !FULL && row >= (uint32_t)a.nrows_full;
-        if (ragged) stage_ragged_row<DTYPE>(stage, (int)t, wv.grad, (uint64_t)row * 32, a.n);
-        read_row_swizzled<DTYPE>(stage, (int)t, x);
-        if (ragged) fence_proxy_async();     // orders those stores before the bulk copy that refills the stage
-    } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) x[j] = 0.0f;
-    }
-    uint32_t m;
-    uint32_t* slot = sh.slots[rot];          // rot = k % 3
-    if constexpr (GIVEN) {
-        m = 0u;
-    } else if constexpr (NORM) {
-        // L2-norm scale: the fixed tree over the rows' sums of squares - partner distance 1, 2, 4, ...
-        // inside the warp, then (buckets of whole warps) the warp sums, one slot per warp
-        float ss = row_sum_squares(x);
-        const uint32_t lanes = SHUFFLE ? a.rows_per_bucket : 32u;
-        for (uint32_t d = 1; d < lanes; d <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xFFFFFFFFu, ss, d));
-        if (!SHUFFLE && (t & 31) == 0) slot[t >> 5] = __float_as_uint(ss);
-        m = __float_as_uint(ss);
-    } else {
-        m = __float_as_uint(row_abs_max(x));
-        if (SHUFFLE) {
-            for (uint32_t d = a.rows_per_bucket >> 1; d > 0; d >>= 1)
-                m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
-        } else {
-            m = __reduce_max_sync(0xFFFFFFFFu, m);
-            if ((t & 31) == 0) atomicMax(&slot[local_bucket], m);
-        }
-    }
-    if (__syncthreads_or(!ok)) return false;
-    if (t == 0) refill(smem_u32(stage), bar);                    // every thread has read the stage
-    if (!SHUFFLE && !GIVEN) {
-        if constexpr (NORM) {
-            // tree over the bucket's warp sums, zero leaves up to four (plain stores: nothing to reset;
-            // the slot array is written again two barriers from here)
-            static_assert(THREADS / 32 == 4, "the warp-sum tree is written for four warps");
-            const uint32_t wpb = a.rows_per_bucket >> 5, first = local_bucket * wpb;
-            float v[4];
-#pragma unroll
-            for (uint32_t i = 0; i < 4; ++i)
-                v[i] = (i < wpb && first + i < 4u) ? __uint_as_float(slot[first + i]) : 0.0f;
-            m = __float_as_uint(__fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3])));
-        } else {
-            m = slot[local_bucket];
-            if (t < THREADS / 32) sh.slots[rot == 0 ? 2 : rot - 1][t] = 0u; // next used by this CTA's tile k + 2
-        }
-    }
-    if (!active) return true;
-
-    float sc = __uint_as_float(m);
-    if constexpr (GIVEN) {
-        sc = __ldg(wv.scales);
-        if (sc < flush_limit()) {        // readers treat the raw and the flushed value alike
-            if (sc != 0.0f && tile == 0 && t == 0) wv.scales[0] = 0.0f;
-            sc = 0.0f;
-        }
-    } else {
-        if constexpr (NORM) sc = sc < flush_limit() ? 0.0f : __fsqrt_rn(sc);     // flush decided on the sum
-        else if (sc < flush_limit()) sc = 0.0f;
-        const uint32_t bucket = tile * a.buckets_per_tile + local_bucket;
-        if (scale_writer && (FULL || bucket < a.nbuckets)) wv.scales[bucket] = sc;
-    }
-
-    const EncodeScale es = encode_scale<BITS>(sc);
-    uint32_t h[16];
-    // Philox blocks of the row: elem_offset / 8 + 4 * row + 0 .. 3, all in the launch's high half
-    draw_row_blocks_head(c.blk0_lo + 4u * row, wv.head, c.rk, h);
-    uint32_t w[BITS];
-    encode_pack_row<BITS>(x, es, h, w);
-    const uint64_t word0 = (uint64_t)row * BITS;
-    if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
-        store_row_words<BITS>(wv.codes, word0, w);
-    } else {
-        mask_row_words<BITS>(w, (int)(a.n - (uint64_t)row * 32) * BITS);
-#pragma unroll
-        for (int j = 0; j < BITS; ++j)
-            if (word0 + j < a.ncode_words) wv.codes[word0 + j] = w[j];
-    }
-    return true;
-}
 
 // The same tile for the (min, max) nearest-rounding variant: two reductions instead of one, two
 // floats per bucket (ranges[2b] = lo, ranges[2b + 1] = hi), no random draws.  Padding must not
@@ -431,7 +223,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_const
     const uint32_t local_bucket = t / a.rows_per_bucket;
     const bool scale_writer = (t % a.rows_per_bucket) == 0;
     const uint32_t ahead = kQuantStages * stride;       // distance to the tile that refills a stage
-    const WorkerView wv = {&tmap, a.grad, a.codes, a.scales, c.head};
+    const WorkerView wv = {&tmap, a.grad, a.codes, a.scales, c.head, c.blk0_lo};
 
     uint32_t k = 0, rot = 0;
     bool ok = true;
@@ -544,7 +336,7 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
 #pragma unroll 1
     for (; ok && v < total_tiles; v += stride, ++k, rot = (rot == 2 ? 0 : rot + 1)) {
         const uint32_t w = cur.w, tile = cur.tile;
-        const WorkerView wv = {&tab.map[w], tab.grad[w], tab.codes[w], tab.scales[w], tab.head[w]};
+        const WorkerView wv = {&tab.map[w], tab.grad[w], tab.codes[w], tab.scales[w], tab.head[w], c.blk0_lo};
         auto refill = [&](uint32_t stage, uint32_t bar) {
             if (vfill < total_tiles) load_tile(fill, stage, bar);
         };
@@ -590,20 +382,22 @@ static cudaError_t launch_tma_inst(const CUtensorMap& map, const QuantizeArgs& a
                                    cudaStream_t stream)
 {
     auto kernel = quantize_tma_kernel<BITS, DTYPE, THREADS, SHUFFLE, MODE>;
-    static int grid_cap[64] = {};                  // per device; 0 = not yet queried
+    static std::atomic<int> grid_cap[64];                  // per device; 0 = not yet queried (zero-initialised)
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (grid_cap[dev] == 0) {
+    int cap = grid_cap[dev].load(std::memory_order_relaxed);
+    if (cap == 0) {
         int occ = 0, sms = 0;
         err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, THREADS, 0);
         if (err != cudaSuccess) return err;
         err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (err != cudaSuccess) return err;
-        grid_cap[dev] = sms * (occ > 0 ? occ : 1);
+        cap = sms * (occ > 0 ? occ : 1);
+        grid_cap[dev].store(cap, std::memory_order_relaxed);   // every thread computes the same value
     }
-    unsigned grid = (unsigned)grid_cap[dev];
+    unsigned grid = (unsigned)cap;
     if (grid > a.ntiles) grid = a.ntiles;
     return launch_pdl(kernel, grid, THREADS, stream, map, a, c, timeouts);
 }
@@ -746,20 +540,22 @@ static cudaError_t launch_workers_inst(const WorkerTable& tab, const QuantizeArg
                                        unsigned int* timeouts, cudaStream_t stream)
 {
     auto kernel = quantize_workers_kernel<BITS, DTYPE, SHUFFLE>;
-    static int grid_cap[64] = {};                  // per device; 0 = not yet queried
+    static std::atomic<int> grid_cap[64];                  // per device; 0 = not yet queried (zero-initialised)
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (grid_cap[dev] == 0) {
+    int cap = grid_cap[dev].load(std::memory_order_relaxed);
+    if (cap == 0) {
         int occ = 0, sms = 0;
         err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, 128, 0);
         if (err != cudaSuccess) return err;
         err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (err != cudaSuccess) return err;
-        grid_cap[dev] = sms * (occ > 0 ? occ : 1);
+        cap = sms * (occ > 0 ? occ : 1);
+        grid_cap[dev].store(cap, std::memory_order_relaxed);   // every thread computes the same value
     }
-    unsigned grid = (unsigned)grid_cap[dev];
+    unsigned grid = (unsigned)cap;
     if (grid > total_tiles) grid = total_tiles;
     return launch_pdl(kernel, grid, 128, stream, tab, a, c, total_tiles, timeouts);
 }

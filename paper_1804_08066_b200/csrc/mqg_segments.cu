@@ -1,7 +1,8 @@
 // Worker side with one scale per segment (per-layer scale) or with buckets larger than a CTA
 // tile: the max and the encode cannot share one pass over on-chip storage, so the gradient
-// is read twice -- a max pass that folds every tile's max into scales[] with an atomic max
-// on the float's bit pattern, then an encode pass identical to the one-pass kernel's.
+// is read twice -- a max pass that folds every tile's max (if it reaches the flush limit) into
+// scales[] with an atomic max on the float's bit pattern, then an encode pass identical to the
+// one-pass kernel's.
 #include "mqg_segments.cuh"
 
 namespace mqg {
@@ -52,7 +53,9 @@ absmax_segments_kernel(const SegQuantArgs a, const SegmentTable tab)
     if (threadIdx.x < 32) {
         m = threadIdx.x < kMaxTileRows / 32 ? s_warp[threadIdx.x] : 0u;
         m = __reduce_max_sync(0xFFFFFFFFu, m);
-        if (threadIdx.x == 0 && m != 0u)
+        // a tile's maximum below the flush limit does not count: a segment whose every tile stays below
+        // it keeps the scale 0 the pass started from, so the scale that stands after the pass is final
+        if (threadIdx.x == 0 && m >= __float_as_uint(flush_limit()))
             atomicMax(reinterpret_cast<unsigned int*>(a.scales) + g.seg, m);
     }
 }
@@ -70,13 +73,7 @@ encode_segments_kernel(const SegQuantArgs a, const SegmentTable tab)
     else
         load_tile_bf16<kMaxTileRows>(tile, static_cast<const uint16_t*>(a.grad) + g.elem0, g.valid, g.rows);
 
-    // the max pass left the raw max; every reader applies the flush, the segment's first tile
-    // also writes it back (readers treat the raw and the flushed value alike)
-    float s = a.scales[g.seg];
-    if (s < flush_limit()) {
-        if (s != 0.0f && g.tile_local == 0 && t == 0) a.scales[g.seg] = 0.0f;
-        s = 0.0f;
-    }
+    const float s = a.scales[g.seg];        // final: the max pass has applied the flush
     __syncthreads();
     if (t >= (uint32_t)g.rows) return;
 

@@ -210,7 +210,11 @@ cudaError_t launch_apply(float* params, const float* acc, float lr, uint64_t n, 
     const uint64_t n4 = n / 4;
     uint64_t blocks = (n4 + 255) / 256;
     if (blocks < 1) blocks = 1;
-    if (blocks > 148ull * 16) blocks = 148ull * 16;
+    int dev = 0, sms = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err == cudaSuccess) err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (err != cudaSuccess) return err;
+    if (blocks > (uint64_t)sms * 16) blocks = (uint64_t)sms * 16;
     apply_kernel<<<(unsigned)blocks, 256, 0, stream>>>(params, acc, lr, n);
     return cudaGetLastError();
 }

@@ -15,6 +15,8 @@
 // A warp therefore never waits for DRAM latency in steady state and there is no CTA-wide barrier
 // anywhere.  Per-(worker, bucket) de-quantization constants are computed once per tile into the
 // warp's small shared table, one tile ahead.
+#include <atomic>
+
 #include "mqg_common.cuh"
 #include "mqg_internal.h"
 #include "mqg_tma.cuh"
@@ -441,12 +443,13 @@ static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, 
 {
     auto kernel = server_tma_kernel<BITS, MODE, RANGE>;
     constexpr size_t kSmemBytes = sizeof(ServerSmem<BITS>) + 1024;   // + slack to round the base up
-    static int grid_cap[64] = {};                 // per device; 0 = not yet set up
+    static std::atomic<int> grid_cap[64];                 // per device; 0 = not yet set up (zero-initialised)
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (grid_cap[dev] == 0) {
+    int cap = grid_cap[dev].load(std::memory_order_relaxed);
+    if (cap == 0) {
         int occ = 0, sms = 0;
         err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (err != cudaSuccess) return err;
@@ -454,10 +457,11 @@ static cudaError_t launch_server_tma_inst(const void* params, ServerTmaArgs& a, 
         if (err != cudaSuccess) return err;
         err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (err != cudaSuccess) return err;
-        grid_cap[dev] = sms * (occ > 0 ? occ : 1);
+        cap = sms * (occ > 0 ? occ : 1);
+        grid_cap[dev].store(cap, std::memory_order_relaxed);   // every thread computes the same value
     }
     // the tiles are split evenly over the warps of the grid; tiny inputs are not spread too thin
-    uint64_t grid = (uint64_t)grid_cap[dev];
+    uint64_t grid = (uint64_t)cap;
     const uint64_t max_warps = (a.ntiles + 3) / 4;
     if (grid * kSrvWarps > max_warps) grid = (max_warps + kSrvWarps - 1) / kSrvWarps;
     CUtensorMap map_full;
