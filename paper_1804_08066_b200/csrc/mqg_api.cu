@@ -622,9 +622,9 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
         if (acc_out && !aligned16(acc_out)) return fail(MQG_ERR_ALIGN, "acc_out not 16-byte aligned");
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    // A long segment is a gradient with a single bucket: it goes to the TMA-fed server kernel in a
-    // launch of its own when its buffers are aligned for bulk copies; all other segments share the
-    // table-driven launch.  The results are the same bit for bit either way.
+    // A long segment is a gradient with a single bucket: the long segments whose buffers are aligned for
+    // bulk copies go to the TMA-fed server kernel together, in one launch; all other segments share
+    // the table-driven launch.  The results are the same bit for bit either way.
     constexpr uint64_t kOwnLaunchElems = 1ull << 20;
     auto own = [&](int j) {
         const uint64_t len = seg_off[j + 1] - seg_off[j];
@@ -641,16 +641,22 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
             return MQG_OK;
         }, own);
     if (st != MQG_OK) return st;
+    // all long segments together, kMaxServerSegsPerLaunch per launch
+    std::vector<mqg::ServerSegHost> longs;
     for (int j = 0; j < nseg; ++j) {
         if (!own(j)) continue;
-        mqg::WorkerPtrs seg_ptrs = ptrs;
-        for (int w = 0; w < W; ++w) {
-            seg_ptrs.codes[w] = codes[w] + code_off[j];
-            seg_ptrs.scales[w] = scales[w] + j;
-        }
-        const uint64_t len = seg_off[j + 1] - seg_off[j];
-        const cudaError_t err = mqg::launch_server(seg_ptrs, W, bits, len, len, params + seg_off[j], lr,
-                                                   nullptr, 0, stream);
+        mqg::ServerSegHost h;
+        h.n = seg_off[j + 1] - seg_off[j];
+        h.elem0 = seg_off[j];
+        h.code_word0 = code_off[j];
+        h.scale_idx = (uint32_t)j;
+        longs.push_back(h);
+    }
+    for (size_t i = 0; i < longs.size(); i += (size_t)mqg::kMaxServerSegsPerLaunch) {
+        const size_t cnt = longs.size() - i < (size_t)mqg::kMaxServerSegsPerLaunch ? longs.size() - i
+                                                                                   : (size_t)mqg::kMaxServerSegsPerLaunch;
+        const cudaError_t err = mqg::launch_server_tma_segments(ptrs, W, bits, longs.data() + i, (int)cnt, params, lr,
+                                                                stream);
         if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
     }
     return MQG_OK;

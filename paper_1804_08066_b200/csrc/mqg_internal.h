@@ -130,6 +130,21 @@ bool server_tma_applies(uint64_t n, uint64_t bucket, int W);   // also buckets o
 cudaError_t launch_server_tma(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
                               float* dst, float lr, int mode, cudaStream_t stream);
 
+// The fused update of up to kMaxServerSegsPerLaunch long segments of a per-layer step in ONE launch of
+// the TMA-fed server kernel (a segment is a gradient with a single bucket).  Every segment must
+// satisfy server_tma_segment_applies(n), and params + elem0 and every worker's codes + code_word0
+// must be 16-byte aligned.
+struct ServerSegHost {
+    uint64_t n;              // elements of the segment
+    uint64_t elem0;          // offset of its first parameter in `params`
+    uint64_t code_word0;     // word offset of its bit stream in every worker's code buffer
+    uint32_t scale_idx;      // index of its scale in every worker's scale array
+};
+constexpr int kMaxServerSegsPerLaunch = 16;
+bool server_tma_segment_applies(uint64_t len);
+cudaError_t launch_server_tma_segments(const WorkerPtrs& ptrs, int W, int bits, const ServerSegHost* segs, int nseg,
+                                       float* params, float lr, cudaStream_t stream);
+
 cudaError_t launch_server_segments(const WorkerPtrs& ptrs, int W, int bits, const SegmentTable& tab,
                                    int scale_base, float* params, float lr, float* acc,
                                    cudaStream_t stream);

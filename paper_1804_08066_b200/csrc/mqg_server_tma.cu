@@ -15,6 +15,8 @@
 // A warp therefore never waits for DRAM latency in steady state and there is no CTA-wide barrier
 // anywhere.  Per-(worker, bucket) de-quantization constants are computed once per tile into the
 // warp's small shared table, one tile ahead.
+#include <string.h>
+
 #include <atomic>
 
 #include "mqg_common.cuh"
@@ -54,6 +56,56 @@ struct ServerTmaArgs {
     uint32_t arm_only;           // test hook: 1 = arm the barriers but issue no parameter copy
 };
 
+// SEGS: the launch covers several gradients ("segments" of a per-layer step, each ONE bucket with a
+// scale of its own) instead of one gradient with uniform buckets.  The tiles of all segments form
+// one sequence that is split over the warps as usual; a tile's segment is found with a cursor that
+// only moves forward.
+constexpr int kMaxSrvSegs = kMaxServerSegsPerLaunch;
+struct ServerSegEntry {
+    uint32_t tile_start;     // number of the segment's first tile in the launch's sequence
+    uint32_t nrows_full;     // floor(n / 32): rows its tensor map and code copies cover
+    uint32_t scale_idx;      // index of its scale in every worker's scale array
+    uint32_t ragged;         // n % 32: elements of its last, incomplete row (0 = none)
+    uint64_t code_word0;     // word offset of its bit stream in every worker's code buffer
+    uint64_t elem0;          // offset of its first element in a.params
+};
+struct ServerSegTable {
+    CUtensorMap map[kMaxSrvSegs];
+    ServerSegEntry e[kMaxSrvSegs + 1];     // e[nseg].tile_start = tiles of the launch
+    int nseg;
+};
+
+// Where a tile lives: the tensor map of its gradient, its first row there, the rows the map covers,
+// the word offset of the gradient's bit stream and (SEGS) the index of its scale.
+struct TileLoc {
+    const CUtensorMap* map;
+    uint32_t row0, nrows_full, scale_idx;
+    uint64_t code_word0;
+};
+
+template <bool SEGS>
+__device__ __forceinline__ TileLoc locate_srv_tile(const CUtensorMap* map_full, const ServerTmaArgs& a,
+                                                   const ServerSegTable* segs, uint32_t tile, uint32_t& cursor)
+{
+    TileLoc t;
+    if constexpr (SEGS) {
+        while (tile >= segs->e[cursor + 1].tile_start) ++cursor;
+        const ServerSegEntry& e = segs->e[cursor];
+        t.map = &segs->map[cursor];
+        t.row0 = (tile - e.tile_start) * kSrvTileRows;
+        t.nrows_full = e.nrows_full;
+        t.scale_idx = e.scale_idx;
+        t.code_word0 = e.code_word0;
+    } else {
+        t.map = map_full;
+        t.row0 = tile * kSrvTileRows;
+        t.nrows_full = a.nrows_full;
+        t.scale_idx = 0;
+        t.code_word0 = 0;
+    }
+    return t;
+}
+
 // Dynamic shared memory of one CTA (base rounded up to 1024 bytes for the 128-byte swizzle).
 template <int BITS>
 struct ServerSmem {
@@ -73,17 +125,18 @@ __device__ __forceinline__ uint32_t bucket_of_row(const ServerTmaArgs& a, uint32
 // when there are more than 32 pairs (`wide`), pair l + 32 (pair = (worker << nbt_shift) +
 // bucket-of-tile).  RANGE: the pair's (lo, hi) instead of its scale (the `scales` pointers then
 // address arrays of two floats per bucket).
-template <bool RANGE>
-__device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, uint32_t row0, uint32_t lane,
+template <bool RANGE, bool SEGS>
+__device__ __forceinline__ void load_tile_scales(const ServerTmaArgs& a, const TileLoc& loc, uint32_t lane,
                                                  bool wide, float2 (&s)[2])
 {
-    const uint32_t first = bucket_of_row(a, row0);
+    // SEGS: the tile lies in one bucket, the segment's (nbt_shift = 0: pair = worker)
+    const uint32_t first = SEGS ? loc.scale_idx : bucket_of_row(a, loc.row0);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         if (h == 1 && !wide) break;
         const uint32_t pair = lane + 32u * h, w = pair >> a.nbt_shift;
         const uint32_t b = first + (pair & ((1u << a.nbt_shift) - 1u));
-        const bool have = w < (uint32_t)a.W && b < a.nbuckets;
+        const bool have = w < (uint32_t)a.W && (SEGS || b < a.nbuckets);
         if (RANGE) s[h] = have ? __ldg(reinterpret_cast<const float2*>(a.ptrs.scales[w]) + b) : make_float2(0.0f, 0.0f);
         else s[h] = make_float2(have ? __ldg(a.ptrs.scales[w] + b) : 0.0f, 0.0f);
     }
@@ -147,18 +200,18 @@ __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.w
 // Starts the copies of one code stage: the words of rows [row0, row0 + 32) (fewer in the last tile
 // of the gradient) of workers g0 .. g0 + group - 1 (those that exist).  A worker's words of these
 // rows are contiguous in its stream and start on a 16-byte boundary (row0 is a multiple of 32):
-// the warp copies them in 16-byte pieces, lane l the l-th piece (and the (l + 32)-th for more than
+// (and so does the bit stream of a segment that takes part in a SEGS launch): the warp copies them in 16-byte pieces, lane l the l-th piece (and the (l + 32)-th for more than
 // four bits), asynchronously and without passing through registers.  The piece that holds the end
 // of a short last tile is copied up to that end and zero-filled.  `lane_off` = 16 * lane.
 template <int BITS>
-__device__ __forceinline__ void fill_code_stage(const ServerTmaArgs& a, uint32_t stage, uint32_t row0, int g0,
+__device__ __forceinline__ void fill_code_stage(const ServerTmaArgs& a, uint32_t stage, const TileLoc& loc, int g0,
                                                 uint32_t lane_off)
 {
     constexpr int kGroup = ServerGroup<BITS>::value;
     constexpr uint32_t kWorkerBytes = kSrvTileRows * BITS * 4;
     constexpr int kPieces = (int)((kWorkerBytes / 16 + 31) / 32);       // pieces per lane: 1 or 2
-    const uint32_t rows_here = min((uint32_t)kSrvTileRows, a.nrows_full - row0);
-    const uint64_t byte0 = (uint64_t)row0 * (BITS * 4) + lane_off;
+    const uint32_t rows_here = min((uint32_t)kSrvTileRows, loc.nrows_full - loc.row0);
+    const uint64_t byte0 = (loc.code_word0 + (uint64_t)loc.row0 * BITS) * 4 + lane_off;
     if (rows_here == (uint32_t)kSrvTileRows && g0 + kGroup <= a.W) {
 #pragma unroll
         for (int pc = 0; pc < kPieces; ++pc) {
@@ -193,10 +246,44 @@ constexpr int server_min_ctas() { return 4; }
 // MODE 1: dst = params, dst <- fma(-lr, sum, dst).  MODE 0: dst = acc, dst <- sum.
 // MODE 2: dst = acc, the sum continues from the value already there.
 // RANGE: the (min, max) nearest-rounding variant (x^ = fma(q, step, lo)).
+// The one row of a gradient that has fewer than 32 elements (row `row`, the last one): plain loads and
+// stores by a single thread.  `params` is the gradient's first parameter, n its length, its bit stream
+// the words [code_word0, words_end) of every worker's buffer, `bucket` the index of the row's scale.
 template <int BITS, int MODE, bool RANGE>
-__global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
-server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ ServerTmaArgs a,
-                  unsigned int* __restrict__ timeouts)
+__device__ __noinline__ void server_ragged_row(const ServerTmaArgs& a, float* params, uint32_t row, uint64_t n,
+                                               uint64_t code_word0, uint64_t words_end, uint32_t bucket)
+{
+    const uint64_t e0 = (uint64_t)row * 32;
+    const uint64_t word0 = code_word0 + (uint64_t)row * BITS;
+    float2 v2[16];
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+        v2[p] = make_float2(0.0f, 0.0f);
+        if constexpr (MODE == 2) {
+            if (e0 + 2 * p < n) v2[p].x = params[e0 + 2 * p];
+            if (e0 + 2 * p + 1 < n) v2[p].y = params[e0 + 2 * p + 1];
+        }
+    }
+    for (int w = 0; w < a.W; ++w) {
+        uint32_t cw[BITS];
+#pragma unroll
+        for (int j = 0; j < BITS; ++j)
+            cw[j] = (word0 + j < words_end) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
+        const DecodeScale2 d = widen(RANGE ? range_decode_scale<BITS>(__ldg(a.ptrs.scales[w] + 2 * bucket),
+                                                                      __ldg(a.ptrs.scales[w] + 2 * bucket + 1))
+                                           : decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
+        add_decoded_row<BITS, RANGE>(cw, d, v2);
+    }
+    float v[32];
+    floats_from_pairs(v2, v);
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        if (e0 + j < n) params[e0 + j] = MODE == 1 ? __fmaf_rn(a.neg_lr, v[j], params[e0 + j]) : v[j];
+}
+
+template <int BITS, int MODE, bool RANGE, bool SEGS>
+__device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, const ServerTmaArgs& a,
+                                                const ServerSegTable* segs, unsigned int* __restrict__ timeouts)
 {
     extern __shared__ uint8_t smem_raw[];
     ServerSmem<BITS>& sm = *reinterpret_cast<ServerSmem<BITS>*>(
@@ -215,7 +302,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     if (lane == 0) {
         mbar_init(bar, 1);
         fence_barrier_init();
-        prefetch_tensormap(&map_full);
+        if (!SEGS) prefetch_tensormap(map_full);
     }
     __syncwarp();
     grid_dependency_wait();            // nothing above touches global memory
@@ -227,8 +314,9 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     const uint32_t base = a.ntiles / nwarps, extra = a.ntiles % nwarps;
     const uint32_t t_begin = gwarp * base + min(gwarp, extra);
     const uint32_t ntiles = base + (gwarp < extra ? 1u : 0u);
-    const uint32_t r_begin = t_begin * kSrvTileRows;
-    const uint32_t last_row = a.nrows_full - 1;    // nrows_full >= 1 on this path
+    const uint32_t last_row = a.nrows_full - 1;    // nrows_full >= 1 on this path (not used by SEGS)
+    uint32_t cur_e = 0, next_e = 0, fill_e = 0;    // SEGS: segment cursors of the tile in work, the next
+                                                   // tile (its scales) and the tile whose codes are fetched
     const uint32_t groups = ((uint32_t)a.W + kGroup - 1) / kGroup;      // code stages per tile
     const uint32_t nunits = ntiles * groups;
     const bool wide = ((uint32_t)a.W << a.nbt_shift) > 32u;             // more than 32 table entries
@@ -243,11 +331,12 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     uint32_t k = 0, u = 0;                         // tile and code stage in use
     if (ntiles > 0) {
         float2 s0[2];
-        load_tile_scales<RANGE>(a, r_begin, lane, wide, s0);
+        const TileLoc first = locate_srv_tile<SEGS>(map_full, a, segs, t_begin, next_e);
+        load_tile_scales<RANGE, SEGS>(a, first, lane, wide, s0);
         store_tile_scales<BITS, RANGE>(a, table, lane, wide, s0);
         if (MODE == 2 && lane == 0) {
             mbar_expect_tx(bar, kSrvTileBytes);
-            if (!a.arm_only) tma_load_2d(smem_u32(stage), &map_full, 0, (int)r_begin, bar);
+            if (!a.arm_only) tma_load_2d(smem_u32(stage), first.map, 0, (int)first.row0, bar);
         }
         // the first kCodeDepth code stages (u2 = stage number, tile u2 / groups, group u2 % groups);
         // one copy group per stage, empty when there is no such stage
@@ -255,7 +344,8 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         for (uint32_t u2 = 0; u2 < (uint32_t)kCodeDepth; ++u2) {
             if (u2 < nunits)
                 fill_code_stage<BITS>(a, code_base + u2 * kCodeStageBytes,
-                                      r_begin + (u2 / groups) * kSrvTileRows, (int)(u2 % groups) * kGroup, lane_off);
+                                      locate_srv_tile<SEGS>(map_full, a, segs, t_begin + u2 / groups, fill_e),
+                                      (int)(u2 % groups) * kGroup, lane_off);
             cp_async_commit();
         }
         __syncwarp();
@@ -266,16 +356,21 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
 #pragma unroll 1
     for (; k < ntiles; ++k) {
         const uint32_t parity = k & 1;
-        const uint32_t row0 = r_begin + k * kSrvTileRows;
+        const TileLoc loc = locate_srv_tile<SEGS>(map_full, a, segs, t_begin + k, cur_e);
+        const uint32_t row0 = loc.row0;
         const bool have_next = k + 1 < ntiles;
         float2 s_next[2];
-        if (have_next) load_tile_scales<RANGE>(a, row0 + kSrvTileRows, lane, wide, s_next);
+        TileLoc loc_next = loc;
+        if (have_next) {
+            loc_next = locate_srv_tile<SEGS>(map_full, a, segs, t_begin + k + 1, next_e);
+            load_tile_scales<RANGE, SEGS>(a, loc_next, lane, wide, s_next);
+        }
 
         // Sum of the W de-quantized rows, in worker order.  Lanes past the end of the gradient
         // (only in the very last tile) decode whatever their slot of the stage holds; they are
         // never stored.
         const uint32_t row = min(row0 + lane, last_row);
-        const uint32_t lb = bucket_of_row(a, row) - bucket_of_row(a, row0);
+        const uint32_t lb = SEGS ? 0u : bucket_of_row(a, row) - bucket_of_row(a, row0);
         const float4* my_table = table + lb;
         float2 v2[16];
         bool ok = true;
@@ -322,7 +417,7 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
                 if (lane == 0) {
                     bulk_wait_read<0>();
                     mbar_expect_tx(bar, kSrvTileBytes);
-                    if (!a.arm_only) tma_load_2d(smem_u32(stage), &map_full, 0, (int)row0, bar);
+                    if (!a.arm_only) tma_load_2d(smem_u32(stage), loc.map, 0, (int)row0, bar);
                 }
             };
             if (g0 + kGroup <= a.W) {              // a whole stage: straight-line code
@@ -341,7 +436,8 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
             }
             __syncwarp();                          // every lane has read the stage: refill it
             if (u + kCodeDepth < nunits)
-                fill_code_stage<BITS>(a, cstage_addr, r_begin + fill_tile * kSrvTileRows,
+                fill_code_stage<BITS>(a, cstage_addr,
+                                      locate_srv_tile<SEGS>(map_full, a, segs, t_begin + fill_tile, fill_e),
                                       (int)fill_group * kGroup, lane_off);
             cp_async_commit();
             if (++fill_group == groups) { fill_group = 0; ++fill_tile; }
@@ -383,12 +479,12 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
         __syncwarp();
         if (lane == 0) {
             // a short last tile is clipped by the tensor's bounds
-            tma_store_2d(&map_full, 0, (int)row0, smem_u32(stage));
+            tma_store_2d(loc.map, 0, (int)row0, smem_u32(stage));
             bulk_commit();
             if (MODE == 2 && have_next) {
                 bulk_wait_read<0>();
                 mbar_expect_tx(bar, kSrvTileBytes);
-                if (!a.arm_only) tma_load_2d(smem_u32(stage), &map_full, 0, (int)(row0 + kSrvTileRows), bar);
+                if (!a.arm_only) tma_load_2d(smem_u32(stage), loc_next.map, 0, (int)loc_next.row0, bar);
             }
         }
     }
@@ -404,37 +500,39 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     }
 
     // A last row of fewer than 32 elements is not covered by the tensor map: one lane of the
-    // grid's last warp handles it with plain loads and stores.
-    if (a.nrows > a.nrows_full && blockIdx.x == gridDim.x - 1 && threadIdx.x == kSrvThreads - 1) {
-        const uint32_t row = a.nrows_full;
-        const uint64_t e0 = (uint64_t)row * 32;
-        const uint64_t word0 = (uint64_t)row * BITS;
-        const uint32_t bucket = bucket_of_row(a, row);
-        float2 v2[16];
-#pragma unroll
-        for (int p = 0; p < 16; ++p) {
-            v2[p] = make_float2(0.0f, 0.0f);
-            if constexpr (MODE == 2) {
-                if (e0 + 2 * p < a.n) v2[p].x = a.params[e0 + 2 * p];
-                if (e0 + 2 * p + 1 < a.n) v2[p].y = a.params[e0 + 2 * p + 1];
+    // grid's last CTA handles it (SEGS: one lane per segment that has such a row).
+    if (blockIdx.x == gridDim.x - 1) {
+        if constexpr (SEGS) {
+            for (int j = (int)threadIdx.x; j < segs->nseg; j += kSrvThreads) {
+                const ServerSegEntry& e = segs->e[j];
+                if (e.ragged == 0) continue;
+                const uint64_t n = (uint64_t)e.nrows_full * 32 + e.ragged;
+                server_ragged_row<BITS, MODE, RANGE>(a, a.params + e.elem0, e.nrows_full, n, e.code_word0,
+                                                     e.code_word0 + (n * BITS + 31) / 32, e.scale_idx);
             }
+        } else if (a.nrows > a.nrows_full && threadIdx.x == kSrvThreads - 1) {
+            server_ragged_row<BITS, MODE, RANGE>(a, a.params, a.nrows_full, a.n, 0, a.ncode_words,
+                                                 bucket_of_row(a, a.nrows_full));
         }
-        for (int w = 0; w < a.W; ++w) {
-            uint32_t cw[BITS];
-#pragma unroll
-            for (int j = 0; j < BITS; ++j)
-                cw[j] = (word0 + j < a.ncode_words) ? __ldg(a.ptrs.codes[w] + word0 + j) : 0u;
-            const DecodeScale2 d = widen(RANGE ? range_decode_scale<BITS>(__ldg(a.ptrs.scales[w] + 2 * bucket),
-                                                                          __ldg(a.ptrs.scales[w] + 2 * bucket + 1))
-                                               : decode_scale<BITS>(__ldg(a.ptrs.scales[w] + bucket)));
-            add_decoded_row<BITS, RANGE>(cw, d, v2);
-        }
-        float v[32];
-        floats_from_pairs(v2, v);
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (e0 + j < a.n) a.params[e0 + j] = MODE == 1 ? __fmaf_rn(a.neg_lr, v[j], a.params[e0 + j]) : v[j];
     }
+}
+
+// One gradient with uniform buckets.
+template <int BITS, int MODE, bool RANGE>
+__global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
+server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_constant__ ServerTmaArgs a,
+                  unsigned int* __restrict__ timeouts)
+{
+    server_tma_body<BITS, MODE, RANGE, false>(&map_full, a, nullptr, timeouts);
+}
+
+// Several long segments of a per-layer step (fused update only).
+template <int BITS>
+__global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
+server_tma_segments_kernel(const __grid_constant__ ServerSegTable segs, const __grid_constant__ ServerTmaArgs a,
+                           unsigned int* __restrict__ timeouts)
+{
+    server_tma_body<BITS, 1, false, true>(nullptr, a, &segs, timeouts);
 }
 
 template <int BITS, int MODE, bool RANGE>
@@ -569,6 +667,94 @@ cudaError_t launch_server_range_tma(const WorkerPtrs& ptrs, int W, int bits, uin
                                     float* params, float lr, int mode, cudaStream_t stream)
 {
     return launch_server_tma_codec<true>(ptrs, W, bits, n, bucket, params, lr, mode, stream);
+}
+
+// ---- several long segments of a per-layer step in one launch --------------------------------------
+template <int BITS>
+static cudaError_t launch_server_segs_inst(const ServerSegTable& tab, const ServerTmaArgs& a, unsigned int* timeouts,
+                                           cudaStream_t stream)
+{
+    auto kernel = server_tma_segments_kernel<BITS>;
+    constexpr size_t kSmemBytes = sizeof(ServerSmem<BITS>) + 1024;   // + slack to round the base up
+    static std::atomic<int> grid_cap[64];                 // per device; 0 = not yet set up (zero-initialised)
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    int cap = grid_cap[dev].load(std::memory_order_relaxed);
+    if (cap == 0) {
+        int occ = 0, sms = 0;
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (err != cudaSuccess) return err;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kSrvThreads, kSmemBytes);
+        if (err != cudaSuccess) return err;
+        err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (err != cudaSuccess) return err;
+        cap = sms * (occ > 0 ? occ : 1);
+        grid_cap[dev].store(cap, std::memory_order_relaxed);   // every thread computes the same value
+    }
+    uint64_t grid = (uint64_t)cap;
+    const uint64_t max_warps = (a.ntiles + 3) / 4;
+    if (grid * kSrvWarps > max_warps) grid = (max_warps + kSrvWarps - 1) / kSrvWarps;
+    return launch_pdl_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, tab, a, timeouts);
+}
+
+bool server_tma_segment_applies(uint64_t len) { return server_tma_applies(len, len); }
+
+cudaError_t launch_server_tma_segments(const WorkerPtrs& ptrs, int W, int bits, const ServerSegHost* segs, int nseg,
+                                       float* params, float lr, cudaStream_t stream)
+{
+    if (nseg < 1 || nseg > kMaxSrvSegs) return cudaErrorInvalidValue;
+    ServerSegTable tab;
+    memset(&tab, 0, sizeof(tab));
+    tab.nseg = nseg;
+    uint64_t tiles = 0;
+    for (int j = 0; j < nseg; ++j) {
+        const ServerSegHost& h = segs[j];
+        ServerSegEntry& e = tab.e[j];
+        const uint64_t nrows_full = h.n / 32;
+        if (nrows_full == 0 || nrows_full > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+        const char* why = nullptr;
+        if (!encode_rows_map(&tab.map[j], params + h.elem0, nrows_full, 4, 32, kSrvTileRows, &why))
+            return cudaErrorNotSupported;
+        e.tile_start = (uint32_t)tiles;
+        e.nrows_full = (uint32_t)nrows_full;
+        e.scale_idx = h.scale_idx;
+        e.ragged = (uint32_t)(h.n % 32);
+        e.code_word0 = h.code_word0;
+        e.elem0 = h.elem0;
+        tiles += (nrows_full + kSrvTileRows - 1) / kSrvTileRows;
+        if (tiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    }
+    tab.e[nseg].tile_start = (uint32_t)tiles;
+    ServerTmaArgs a;
+    memset(&a, 0, sizeof(a));
+    a.ptrs = ptrs;
+    a.params = params;
+    a.nrows = a.nrows_full = 1;          // not used by a launch over segments
+    a.ntiles = (uint32_t)tiles;
+    a.nbuckets = 1;
+    a.rows_per_bucket = 1; a.rpb_shift = 0;
+    a.nbt_shift = 0;                     // a tile lies in one bucket: table entry = worker
+    a.W = W;
+    a.neg_lr = -lr;
+    a.bias_bits = 0x4B000000u;
+    const WaitPolicy policy = wait_policy();
+    a.poll_limit = policy.poll_limit;
+    a.arm_only = policy.arm_only;
+    unsigned int* timeouts = wait_timeout_counter();
+    if (timeouts == nullptr) return cudaErrorNotSupported;
+    switch (bits) {
+        case 1: return launch_server_segs_inst<1>(tab, a, timeouts, stream);
+        case 2: return launch_server_segs_inst<2>(tab, a, timeouts, stream);
+        case 3: return launch_server_segs_inst<3>(tab, a, timeouts, stream);
+        case 4: return launch_server_segs_inst<4>(tab, a, timeouts, stream);
+        case 5: return launch_server_segs_inst<5>(tab, a, timeouts, stream);
+        case 6: return launch_server_segs_inst<6>(tab, a, timeouts, stream);
+        case 7: return launch_server_segs_inst<7>(tab, a, timeouts, stream);
+        case 8: return launch_server_segs_inst<8>(tab, a, timeouts, stream);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace mqg
