@@ -528,7 +528,7 @@ def run_ours(args):
     sm_clock_hz = (clocks.summary().get("sm_mhz") or 1965.0) * 1e6
     alu_peak = 148 * 128 * sm_clock_hz / 1e9
     alu_achieved = (4 * W + 13) * n / (down_us * 1e-6) / 1e9
-    downlink_line = {"kernel": "requantize_kernel (mqg_server_requantize, all bit widths, not part of `value`)",
+    downlink_line = {"kernel": "requantize_warp_kernel (mqg_server_requantize, all bit widths, not part of `value`)",
                      "avg_launch_us": down_us, "grad_gbs": 4 * n * W / (down_us * 1e-6) / 1e9,
                      "roofline": {"bound": "alu", "achieved": alu_achieved, "peak": alu_peak,
                                   "unit": "G lane-op/s", "frac": alu_achieved / alu_peak, "traffic": None,

@@ -154,6 +154,12 @@ cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
                               float mean_scale, uint64_t seed, uint32_t* codes_out, float* scales_out,
                               uint32_t worker, uint32_t step, cudaStream_t stream);
 
+// The same on the warp-pipelined kernel of mqg_server_tma.cu (whole rows, buckets of 2^k rows up to 128).
+bool requantize_warp_applies(uint64_t n, uint64_t bucket, int W);
+cudaError_t launch_requantize_warp(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                                   float mean_scale, uint64_t seed, uint32_t* codes_out, float* scales_out,
+                                   uint32_t worker, uint32_t step, cudaStream_t stream);
+
 cudaError_t launch_apply(float* params, const float* acc, float lr, uint64_t n, cudaStream_t stream);
 
 }  // namespace mqg

@@ -207,6 +207,9 @@ cudaError_t launch_requantize(const WorkerPtrs& ptrs, int W, int bits, uint64_t 
                               float mean_scale, uint64_t seed, uint32_t* codes_out, float* scales_out,
                               uint32_t worker, uint32_t step, cudaStream_t stream)
 {
+    if (requantize_warp_applies(n, bucket, W))
+        return launch_requantize_warp(ptrs, W, bits, n, bucket, mean_scale, seed, codes_out, scales_out, worker, step,
+                                      stream);
     RequantArgs a;
     a.ptrs = ptrs; a.codes_out = codes_out; a.scales_out = scales_out;
     a.n = n;

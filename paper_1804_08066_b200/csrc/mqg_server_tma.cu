@@ -669,6 +669,269 @@ cudaError_t launch_server_range_tma(const WorkerPtrs& ptrs, int W, int bits, uin
     return launch_server_tma_codec<true>(ptrs, W, bits, n, bucket, params, lr, mode, stream);
 }
 
+// ---- downlink: de-quantize, sum, scale to the mean and quantize again -------------------------------
+// (ReceiveQGThenSendQG of Algorithm 1, lines 1-5; steps 6-8 of Fig. 3.)  The decode half is the server
+// kernel's: every warp stages the code words of its 32-row tiles by asynchronous copies, two stages
+// ahead, and sums the W workers in registers.  The encode half is the quantize kernels' row code.  In
+// between stands the bucket maximum: a CTA takes 128 consecutive rows at a time, one 32-row tile per
+// warp, so a bucket of 32 rows or fewer is reduced by lane shuffles and a bucket of 64 or 128 rows by
+// the two or four warps that hold it, through shared memory and a named barrier of just those warps.
+// Persistent CTAs, no CTA-wide barrier, no global load through registers.
+struct RequantWarpArgs {
+    ServerTmaArgs s;             // decode side: ptrs, nrows_full (= all rows), buckets, W, bias
+    uint32_t* codes_out;
+    float* scales_out;
+    float mean_scale;
+    uint32_t nct;                // CTA tiles of 128 rows
+    uint32_t warps_per_bucket;   // 1 (buckets of at most 32 rows), 2 or 4
+    RoundKeys rk;                // Philox round keys of the re-quantization's draws
+    PhiloxHead head;             // and the launch-wide part of its blocks
+};
+
+template <int BITS>
+struct RequantSmem {
+    alignas(16) uint32_t code[kSrvWarps][kCodeDepth][ServerGroup<BITS>::value][kSrvTileRows * BITS];
+    float4 table[kSrvWarps][2 * kMaxWorkers];
+    uint32_t bmax[2][kSrvWarps];                  // tile maxima, double-buffered by the parity of the turn
+};
+
+template <int ID>
+__device__ __forceinline__ void named_barrier(uint32_t threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "r"(threads) : "memory");
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kSrvThreads, 4)
+requantize_warp_kernel(const __grid_constant__ RequantWarpArgs ra)
+{
+    extern __shared__ uint8_t smem_raw[];
+    RequantSmem<BITS>& sm = *reinterpret_cast<RequantSmem<BITS>*>(
+        smem_raw + ((16u - (smem_u32(smem_raw) & 15u)) & 15u));
+    const ServerTmaArgs& a = ra.s;
+    constexpr int kGroup = ServerGroup<BITS>::value;
+    constexpr uint32_t kWorkerWords = kSrvTileRows * BITS;
+    constexpr uint32_t kCodeStageBytes = kGroup * kWorkerWords * 4;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t wid = __shfl_sync(0xFFFFFFFFu, threadIdx.x >> 5, 0);
+    float4* table = sm.table[wid];
+    const uint32_t code_base = smem_u32(&sm.code[wid][0][0][0]);
+    grid_dependency_wait();            // nothing above touches global memory
+
+    // this CTA's tiles of 128 rows: [ct_begin, ct_begin + nct); warp w takes rows 32 w .. 32 w + 31 of each
+    const uint32_t base = ra.nct / gridDim.x, extra = ra.nct % gridDim.x;
+    const uint32_t ct_begin = blockIdx.x * base + min(blockIdx.x, extra);
+    const uint32_t nct = base + (blockIdx.x < extra ? 1u : 0u);
+    const uint32_t groups = ((uint32_t)a.W + kGroup - 1) / kGroup;      // code stages per tile
+    const uint32_t nunits = nct * groups;
+    const bool wide = ((uint32_t)a.W << a.nbt_shift) > 32u;
+    const uint32_t lane_off = lane * 16u;
+    const uint32_t last_row = a.nrows_full - 1;
+    const uint32_t G = ra.warps_per_bucket;
+    auto tile_loc = [&](uint32_t kk) {
+        TileLoc t;
+        t.map = nullptr;
+        t.row0 = ((ct_begin + kk) * kSrvWarps + wid) * kSrvTileRows;
+        t.nrows_full = a.nrows_full;
+        t.scale_idx = 0;
+        t.code_word0 = 0;
+        return t;
+    };
+    auto fill = [&](uint32_t stage, uint32_t kk, int g0) {           // a tile beyond the last row has no codes
+        const TileLoc t = tile_loc(kk);
+        if (t.row0 < a.nrows_full) fill_code_stage<BITS>(a, stage, t, g0, lane_off);
+    };
+
+    uint32_t u = 0;
+    if (nct > 0) {
+        float2 s0[2];
+        load_tile_scales<false, false>(a, tile_loc(0), lane, wide, s0);
+        store_tile_scales<BITS, false>(a, table, lane, wide, s0);
+#pragma unroll
+        for (uint32_t u2 = 0; u2 < (uint32_t)kCodeDepth; ++u2) {
+            if (u2 < nunits) fill(code_base + u2 * kCodeStageBytes, u2 / groups, (int)(u2 % groups) * kGroup);
+            cp_async_commit();
+        }
+        __syncwarp();
+    }
+    uint32_t fill_tile = kCodeDepth / groups, fill_group = kCodeDepth % groups;
+
+#pragma unroll 1
+    for (uint32_t k = 0; k < nct; ++k) {
+        const TileLoc loc = tile_loc(k);
+        const uint32_t row0 = loc.row0;
+        const bool have_next = k + 1 < nct;
+        float2 s_next[2];
+        if (have_next) load_tile_scales<false, false>(a, tile_loc(k + 1), lane, wide, s_next);
+        const uint32_t row_c = min(row0 + lane, last_row);
+        const uint32_t lb = bucket_of_row(a, row_c) - bucket_of_row(a, min(row0, last_row));
+        const float4* my_table = table + lb;
+        float2 v2[16];
+#pragma unroll
+        for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
+
+#pragma unroll 1
+        for (uint32_t g = 0; g < groups; ++g, ++u) {
+            const uint32_t cs = u % kCodeDepth;
+            const uint32_t* cstage = &sm.code[wid][cs][0][0] + lane * BITS;
+            cp_async_wait_group<kCodeDepth - 1>();
+            __syncwarp();
+            const int g0 = (int)g * kGroup;
+            auto decode_worker = [&](int i) {
+                uint32_t w[BITS];
+                read_stage_words<BITS>(cstage + i * kWorkerWords, w);
+                const float4 e = my_table[(uint32_t)(g0 + i) << a.nbt_shift];
+                DecodeScale2 d;
+                d.two_h = make_float2(e.x, e.y); d.minus_h = make_float2(e.z, e.w);
+                add_decoded_row<BITS, false>(w, d, v2, a.bias_bits);
+            };
+            if (g0 + kGroup <= a.W) {
+#pragma unroll
+                for (int i = 0; i < kGroup; ++i) decode_worker(i);
+            } else {
+#pragma unroll 1
+                for (int i = 0; g0 + i < a.W; ++i) decode_worker(i);
+            }
+            __syncwarp();                          // every lane has read the stage: refill it
+            if (u + kCodeDepth < nunits) fill(code_base + cs * kCodeStageBytes, fill_tile, (int)fill_group * kGroup);
+            cp_async_commit();
+            if (++fill_group == groups) { fill_group = 0; ++fill_tile; }
+        }
+
+        // the mean, and the bucket maximum of its magnitudes
+        const uint32_t row = row0 + lane;
+        const bool active = row < a.nrows_full;
+        float x[32];
+        {
+            const float2 ms = make_float2(ra.mean_scale, ra.mean_scale);
+#pragma unroll
+            for (int p = 0; p < 16; ++p) {
+                const float2 y = __fmul2_rn(v2[p], ms);
+                x[2 * p] = y.x;
+                x[2 * p + 1] = y.y;
+            }
+            if (row0 + kSrvTileRows > a.nrows_full && !active) {     // only in the gradient's last tiles:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = 0.0f;            // lanes past the end decode what their slot holds
+            }
+        }
+        uint32_t m = __float_as_uint(row_abs_max(x));
+        if (G == 1) {
+            const uint32_t rpb = min(a.rows_per_bucket, (uint32_t)kSrvTileRows);
+            for (uint32_t d = rpb >> 1; d > 0; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+        } else {
+            m = __reduce_max_sync(0xFFFFFFFFu, m);
+            uint32_t* slot = sm.bmax[k & 1];
+            if (lane == 0) slot[wid] = m;
+            const uint32_t first = wid & ~(G - 1);
+            if (G == 4 || first == 0) named_barrier<1>(32 * G);   // the warps that hold this bucket
+            else named_barrier<2>(32 * G);
+            m = max(slot[first], slot[first + 1]);
+            if (G == 4) m = max(m, max(slot[first + 2], slot[first + 3]));
+        }
+        float sc = __uint_as_float(m);
+        if (sc < flush_limit()) sc = 0.0f;
+        if (active) {
+            const bool writer = G == 1 ? (row & (a.rows_per_bucket - 1)) == 0 : ((wid & (G - 1)) == 0 && lane == 0);
+            if (writer) ra.scales_out[row >> a.rpb_shift] = sc;
+            const EncodeScale es = encode_scale<BITS>(sc);
+            // (spreading the four Philox blocks over the decode of the workers, to fill its gaps, measured
+            // 3 to 5 us slower per launch: the kernel then needs all 128 registers)
+            uint32_t h[16];
+            draw_row_blocks_head(4u * row, ra.head, ra.rk, h);     // the downlink draws from position 0
+            uint32_t w[BITS];
+            encode_pack_row<BITS>(x, es, h, w);
+            store_row_words<BITS>(ra.codes_out, (uint64_t)row * BITS, w);
+        }
+        if (have_next) store_tile_scales<BITS, false>(a, table, lane, wide, s_next);
+        __syncwarp();
+    }
+    cp_async_wait_group<0>();                                  // no code copy outlives the warp
+}
+
+template <int BITS>
+static cudaError_t launch_requantize_warp_inst(const RequantWarpArgs& ra, cudaStream_t stream)
+{
+    auto kernel = requantize_warp_kernel<BITS>;
+    constexpr size_t kSmemBytes = sizeof(RequantSmem<BITS>) + 16;
+    static std::atomic<int> grid_cap[64];                 // per device; 0 = not yet set up (zero-initialised)
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    int cap = grid_cap[dev].load(std::memory_order_relaxed);
+    if (cap == 0) {
+        int occ = 0, sms = 0;
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (err != cudaSuccess) return err;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kSrvThreads, kSmemBytes);
+        if (err != cudaSuccess) return err;
+        err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (err != cudaSuccess) return err;
+        cap = sms * (occ > 0 ? occ : 1);
+        grid_cap[dev].store(cap, std::memory_order_relaxed);   // every thread computes the same value
+    }
+    unsigned grid = (unsigned)cap;
+    if (grid > ra.nct) grid = ra.nct;
+    return launch_pdl_smem(kernel, grid, kSrvThreads, kSmemBytes, stream, ra);
+}
+
+// Whole rows, at least 512 of them, fewer than 2^30 (so the draws' block numbers have no high half),
+// and buckets of 2^k rows, k <= 7 (at most 4096 elements), those below 32 rows few enough per tile for
+// the warp's table.
+bool requantize_warp_applies(uint64_t n, uint64_t bucket, int W)
+{
+    if (n % 32 != 0 || n / 32 < 512 || n / 32 >= (1ull << 30) || bucket >= n || bucket % 32 != 0) return false;
+    const uint64_t rpb = bucket / 32;
+    if ((rpb & (rpb - 1)) != 0 || rpb > 128) return false;
+    if (rpb >= 32) return true;
+    return ((uint64_t)W * (32 / rpb)) <= 2 * (uint64_t)kMaxWorkers;
+}
+
+cudaError_t launch_requantize_warp(const WorkerPtrs& ptrs, int W, int bits, uint64_t n, uint64_t bucket,
+                                   float mean_scale, uint64_t seed, uint32_t* codes_out, float* scales_out,
+                                   uint32_t worker, uint32_t step, cudaStream_t stream)
+{
+    RequantWarpArgs ra;
+    memset(&ra, 0, sizeof(ra));
+    ServerTmaArgs& a = ra.s;
+    a.ptrs = ptrs;
+    a.n = n;
+    a.ncode_words = (n * (uint64_t)bits + 31) / 32;
+    a.nrows = a.nrows_full = (uint32_t)(n / 32);
+    a.nbuckets = (uint32_t)((n + bucket - 1) / bucket);
+    const uint64_t rpb = bucket / 32;
+    a.rows_per_bucket = (uint32_t)rpb;
+    a.rpb_shift = 0;
+    while (((uint64_t)1 << a.rpb_shift) < rpb) ++a.rpb_shift;
+    a.nbt_shift = 0;                                     // buckets a tile of 32 rows touches: 32 / rpb
+    while (rpb < 32 && (rpb << a.nbt_shift) < 32) ++a.nbt_shift;
+    a.W = W;
+    a.bias_bits = 0x4B000000u;
+    ra.codes_out = codes_out; ra.scales_out = scales_out;
+    ra.mean_scale = mean_scale;
+    ra.nct = (uint32_t)((n / 32 + kSrvThreads - 1) / kSrvThreads);
+    ra.warps_per_bucket = rpb <= 32 ? 1u : (uint32_t)(rpb / 32);
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        ra.rk.k0[r] = k0; ra.rk.k1[r] = k1;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    ra.rk.worker = worker; ra.rk.step = step;
+    ra.head = philox_head(0u, worker, ra.rk.k0[0]);
+    switch (bits) {
+        case 1: return launch_requantize_warp_inst<1>(ra, stream);
+        case 2: return launch_requantize_warp_inst<2>(ra, stream);
+        case 3: return launch_requantize_warp_inst<3>(ra, stream);
+        case 4: return launch_requantize_warp_inst<4>(ra, stream);
+        case 5: return launch_requantize_warp_inst<5>(ra, stream);
+        case 6: return launch_requantize_warp_inst<6>(ra, stream);
+        case 7: return launch_requantize_warp_inst<7>(ra, stream);
+        case 8: return launch_requantize_warp_inst<8>(ra, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
 // ---- several long segments of a per-layer step in one launch --------------------------------------
 template <int BITS>
 static cudaError_t launch_server_segs_inst(const ServerSegTable& tab, const ServerTmaArgs& a, unsigned int* timeouts,

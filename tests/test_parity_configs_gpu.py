@@ -152,3 +152,27 @@ def test_billion_element_bf16_stress_sampled(bits):
         O.server_step([host[(k, w)][0] for w in order], [host[(k, w)][1] for w in order], bits, hi - lo, B, p_ref, 0.01)
         assert bits_equal(params[lo:hi].cpu().numpy(), p_ref) == 0, k
     assert mqg.mqg_device_timeouts() == 0
+
+
+@pytest.mark.parametrize("bits", [3, 8])
+def test_batched_bf16_bucket_4096_four_workers(bits):
+    """The stress shape's kernel instantiation (bf16 input widened in the kernel, bucket 4096) in the
+    batched launch, 4 workers x (2^26 + 2560) elements (16,385 buckets per worker, the last one short),
+    every element of every worker against the CPU checker."""
+    from concurrent.futures import ThreadPoolExecutor
+    n, B, W = (1 << 26) + 2560, 4096, 4
+    with ThreadPoolExecutor(W) as ex:
+        xs = list(ex.map(lambda w: wl.student_t_bf16(n, config=5, worker=w), range(W)))
+        refs = list(ex.map(lambda w: O.quantize(xs[w], bits, B, 6, worker=10 + w, step=2, elem_offset=1 << 20,
+                                                dtype="bf16"), range(W)))
+    grads = [to_dev(x.view(np.int16)).view(torch.bfloat16) for x in xs]
+    codes = [Guarded(mqg.mqg_code_words(n, bits), torch.int32) for _ in range(W)]
+    scales = [Guarded(mqg.mqg_num_buckets(n, B), torch.float32) for _ in range(W)]
+    mqg.mqg_quantize_workers(grads, W, n, bits, B, 6, [c.view for c in codes], [s.view for s in scales],
+                             first_worker=10, step=2, elem_offset=1 << 20)
+    torch.cuda.synchronize()
+    for w in range(W):
+        codes[w].check_guards(), scales[w].check_guards()
+        assert bits_equal(scales[w].numpy(np.float32), refs[w][1]) == 0, w
+        assert np.array_equal(codes[w].numpy(np.uint32), refs[w][0]), w
+    assert mqg.mqg_device_timeouts() == 0

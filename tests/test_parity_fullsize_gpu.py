@@ -1,6 +1,7 @@
 """Parity at the benchmark's full size and launch configuration: n = 25,000,000 fp32 per
 worker, W = 8, Laplace(0, 1e-4), bucket 2048 (12,207 full buckets and one of 64 elements),
-every bit width, checked element by element against the CPU checker."""
+every bit width, checked element by element against the CPU checker - with one launch per worker
+and with the one batched launch for all workers that the benchmark times."""
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -45,6 +46,21 @@ def test_full_size_step(bits):
         if not np.array_equal(got, ref[w][0]):
             differing += int((O.unpack(got, N, bits) != O.unpack(ref[w][0], N, bits)).sum())
         codes.append(dc), scales.append(ds)
+    # the launch the benchmark times: all eight gradients in ONE mqg_quantize_workers launch (48,832
+    # tiles walked as one sequence); the server step below reads what this launch wrote
+    del codes, scales
+    bc = [Guarded(mqg.mqg_code_words(N, bits), torch.int32) for _ in range(W)]
+    bs = [Guarded(mqg.mqg_num_buckets(N, B), torch.float32) for _ in range(W)]
+    mqg.mqg_quantize_workers(c["dev"], W, N, bits, B, SEED, [d.view for d in bc], [d.view for d in bs],
+                             first_worker=0, step=7)
+    torch.cuda.synchronize()
+    for w in range(W):
+        bc[w].check_guards(), bs[w].check_guards()
+        assert bits_equal(bs[w].numpy(np.float32), ref[w][1]) == 0, w
+        got = bc[w].numpy(np.uint32)
+        if not np.array_equal(got, ref[w][0]):
+            differing += int((O.unpack(got, N, bits) != O.unpack(ref[w][0], N, bits)).sum())
+    codes, scales = bc, bs
     # the stated bar allows threshold ties up to 1e-6 of n; none are expected
     assert differing <= 1e-6 * N * W
     assert differing == 0

@@ -341,7 +341,13 @@ def test_segments_more_than_one_launch_chunk():
 # ------------------------------------------------------------------ downlink: server re-quantization
 @pytest.mark.parametrize("bits", ALL_BITS)
 @pytest.mark.parametrize("n,bucket,W", [(40, 64, 1), (8192 + 5, 2048, 3), (100_003, 4096, 4), (9000, 96, 2),
-                                        (5000, 10_000 - 1808, 5), (65_536 + 31, 512, 8)])
+                                        (5000, 10_000 - 1808, 5), (65_536 + 31, 512, 8),
+                                        # whole rows, power-of-two buckets: the warp-pipelined kernel (buckets
+                                        # held by two warps, four warps, one warp, parts of a warp; short last
+                                        # buckets; worker counts that do not fill a code stage; 32 workers)
+                                        ((1 << 17) + 64, 2048, 8), ((1 << 17) + 5 * 1024, 4096, 3), (99_968, 1024, 5),
+                                        (32_768 + 64, 256, 8), (16_384 + 32, 32, 2), (22_400, 64, 4),
+                                        (1 << 15, 2048, 32), ((1 << 16) + 2048 + 32, 2048, 9)])
 def test_server_requantize(bits, n, bucket, W):
     xs = [wl.normal(n, 2e-3, config=41, worker=w) for w in range(W)]
     if n >= bucket:
