@@ -52,9 +52,13 @@ METRIC = "quantize+pack and dequant+accumulate+update GB/s (fp32 grad) per bit w
 UNIT = "GB/s of fp32 gradient through quantize+pack -> unpack+accumulate+update"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per element of quantize_workers_kernel<4> (ncu, 4 x 8,388,608
-# elements): (134.25 MB + 7.82 MB) / 33,554,432; writes are partly still in L2 when the kernel ends
-QUANTIZE_DRAM_BYTES_PER_ELEM_K4 = 142.48e6 / 33_554_432
+# dram__bytes_read.sum + dram__bytes_write.sum per element and bit width, from the ncu captures on small
+# cases summarised in profiles/per_width_counters_small_cases.md (quantize_workers_kernel: 4 x 8,388,608
+# elements; server_tma_kernel: n = 2^25, W = 8; both bucket 2048).  DRAM traffic grows in proportion to the
+# elements, so a launch's traffic is the figure times its elements.  Writes are partly still in L2 when a
+# kernel ends, hence less than the algorithmic bytes (4 + K/8 and 8 + W K/8 per element).
+QUANTIZE_DRAM_BYTES_PER_ELEM = {1: 4.0771, 2: 4.1061, 3: 4.141, 4: 4.2012, 5: 4.2161, 6: 4.2546, 7: 4.3087, 8: 4.3646}
+SERVER_DRAM_BYTES_PER_ELEM = {1: 7.2747, 2: 8.3364, 3: 9.4213, 4: 10.4596, 5: 11.6609, 6: 12.7271, 7: 13.795, 8: 14.8942}
 
 
 def measured_hbm_peak():
@@ -192,9 +196,16 @@ def cpu_baseline(grads, target_seconds=20.0):
     n_s = max(BUCKET, min(N_ELEMS // BUCKET * BUCKET, n_s // BUCKET * BUCKET))
     secs = oracle_pass(grads, n_s, ALL_BITS, threads)
     gbs = len(ALL_BITS) * len(grads) * 4 * n_s / secs / 1e9
+    # the same checker on ONE host thread (the definition's own speed), on a sample 1/32 the size
+    n_1 = max(BUCKET, n_s // 32 // BUCKET * BUCKET)
+    secs_1 = oracle_pass(grads, n_1, ALL_BITS, 1)
+    gbs_1 = len(ALL_BITS) * len(grads) * 4 * n_1 / secs_1 / 1e9
     return {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": "first %d of %d elements of each of %d workers, bits 1..8, one pass in %.2f s"
-                      % (n_s, N_ELEMS, len(grads), secs)}, n_s
+                      % (n_s, N_ELEMS, len(grads), secs),
+            "single_thread": {"value": gbs_1, "cores": 1,
+                              "sample": "first %d elements of each of %d workers, bits 1..8, one pass in %.2f s"
+                                        % (n_1, len(grads), secs_1)}}, n_s
 
 
 def run_reference(args):
@@ -479,6 +490,8 @@ def run_ours(args):
             "server_us_best": min(s_ms[b]) * 1e3,
             "server_us_single_median": float(np.median(s_single[b])) * 1e3,
             "server_us_single_best": min(s_single[b]) * 1e3,
+            "quantize_dram_traffic": QUANTIZE_DRAM_BYTES_PER_ELEM[b] * n, "quantize_algorithmic_bytes": qb,
+            "server_dram_traffic": SERVER_DRAM_BYTES_PER_ELEM[b] * n, "server_algorithmic_bytes": sb,
             "wire_bytes_per_worker": mqg.mqg_wire_bytes(n, b, B),
             ("quantize_us_per_worker_launches" if batched else "quantize_us_one_launch"): other_ms[b] / W * 1e3,
         })
@@ -493,16 +506,21 @@ def run_ours(args):
                 "bound": "hbm", "achieved": q_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
                 "unit": "GB/s", "frac": q_achieved / peak,
                 "avg_launch_us": q_phase_s / (len(ALL_BITS) * q_launches) * 1e6,
-                "traffic": QUANTIZE_DRAM_BYTES_PER_ELEM_K4 * n * q_per_launch,
-                "traffic_note": "dram read+write bytes per element of a K=4 launch from the ncu capture in "
-                                "profiles/quantize_workers_kernel_b4_W4_n8M.md (33.5M elements; both quantize "
-                                "kernels run the same tile code), scaled to the elements of one launch; "
-                                "algorithmic bytes of that launch: %d" % (quantize_bytes(n, 4, B) * q_per_launch),
+                "traffic": float(np.mean([QUANTIZE_DRAM_BYTES_PER_ELEM[b] for b in ALL_BITS])) * n * q_per_launch,
+                "traffic_note": "dram read+write bytes per launch, mean over the eight bit widths of the phase "
+                                "(`per_bits[].quantize_dram_traffic` has each width), from the ncu captures of "
+                                "profiles/per_width_counters_small_cases.md scaled to the elements of one launch; "
+                                "algorithmic bytes of a launch, same mean: %d"
+                                % int(np.mean([quantize_bytes(n, b, B) for b in ALL_BITS]) * q_per_launch),
                 "time_share_of_step": q_time_total / (q_time_total + s_time_total)}
     roofline_server = {"kernel": "server_tma_kernel (fused step, all bit widths, %d launches per step)" % len(ALL_BITS),
                        "bound": "hbm", "achieved": s_achieved, "peak": peak, "peak_kind": peak_kind + " copy rate",
                        "unit": "GB/s", "frac": s_achieved / peak,
-                       "avg_launch_us": s_phase_s / len(ALL_BITS) * 1e6, "traffic": None}
+                       "avg_launch_us": s_phase_s / len(ALL_BITS) * 1e6,
+                       "traffic": float(np.mean([SERVER_DRAM_BYTES_PER_ELEM[b] for b in ALL_BITS])) * n,
+                       "traffic_note": "dram read+write bytes per launch, mean over the eight bit widths (each "
+                                       "width: `per_bits[].server_dram_traffic`), same source; algorithmic: %d"
+                                       % int(np.mean([server_bytes(n, b, B, W) for b in ALL_BITS]))}
 
     # ---- the downlink (outside `value`): the server re-quantizes the mean for the broadcast.  ALU-bound:
     # per element 4 W + 13 lane operations (per worker 1 extract + 3 fp for the decode and sum; mean, max,

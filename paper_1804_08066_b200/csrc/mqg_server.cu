@@ -35,16 +35,30 @@ __device__ __forceinline__ void accumulate_row(const ServerArgs& a, uint64_t sca
 #pragma unroll
         for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
     }
-    for (int wk = 0; wk < a.W; ++wk) {
-        uint32_t w[BITS];
-        if (VEC && full_row) load_row_words<BITS>(a.ptrs.codes[wk], word0, w);
-        else {
+    // four workers at a time: their code words and scales are all requested before the first one is
+    // decoded, so that a row waits for global memory once per four workers, not once per worker
+    constexpr int kBatch = 4;
+    for (int w0 = 0; w0 < a.W; w0 += kBatch) {
+        uint32_t w[kBatch][BITS];
+        float sc[kBatch];
 #pragma unroll
-            for (int k = 0; k < BITS; ++k)
-                w[k] = (word0 + k < words_end) ? __ldg(a.ptrs.codes[wk] + word0 + k) : 0u;
+        for (int i = 0; i < kBatch; ++i) {
+            const int wk = min(w0 + i, a.W - 1);            // a worker past the last one repeats it (not summed)
+            if (VEC && full_row) load_row_words<BITS>(a.ptrs.codes[wk], word0, w[i]);
+            else {
+#pragma unroll
+                for (int k = 0; k < BITS; ++k)
+                    w[i][k] = (word0 + k < words_end) ? __ldg(a.ptrs.codes[wk] + word0 + k) : 0u;
+            }
+            sc[i] = __ldg(a.ptrs.scales[wk] + scale_idx);
         }
-        const DecodeScale2 d = widen(decode_scale<BITS>(__ldg(a.ptrs.scales[wk] + scale_idx)));
-        add_decoded_row<BITS>(w, d, v2);
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            if (w0 + i < a.W) {
+                const DecodeScale2 d = widen(decode_scale<BITS>(sc[i]));
+                add_decoded_row<BITS>(w[i], d, v2);
+            }
+        }
     }
     floats_from_pairs(v2, v);
 }
