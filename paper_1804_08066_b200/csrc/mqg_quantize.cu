@@ -333,22 +333,29 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
 
     uint32_t k = 0, rot = 0;
     bool ok = true;
+    uint32_t w = cur.w, tile = cur.tile;
+    // Outer loop: the workers this CTA's walk passes through; inner loop: its tiles of that worker.  The
+    // worker's table entries (pointers, Philox head) are fetched once per worker, not once per tile:
+    // indexed loads from the kernel's parameter block are long-latency loads the tile would wait for.
 #pragma unroll 1
-    for (; ok && v < total_tiles; v += stride, ++k, rot = (rot == 2 ? 0 : rot + 1)) {
-        const uint32_t w = cur.w, tile = cur.tile;
+    while (ok && v < total_tiles) {
         const WorkerView wv = {&tab.map[w], tab.grad[w], tab.codes[w], tab.scales[w], tab.head[w], c.blk0_lo};
-        auto refill = [&](uint32_t stage, uint32_t bar) {
-            if (vfill < total_tiles) load_tile(fill, stage, bar);
-        };
-        if (tile < c.full_tiles)
-            ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, rot, tile, refill,
-                                                                     local_bucket, scale_writer);
-        else
-            ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, rot, tile, refill,
-                                                                      local_bucket, scale_writer);
-        if (v + stride < total_tiles) advance(cur, stride);
-        vfill += stride;
-        if (vfill < total_tiles) advance(fill, stride);
+#pragma unroll 1
+        for (; ok && tile < a.ntiles && v < total_tiles;
+             tile += stride, v += stride, ++k, rot = (rot == 2 ? 0 : rot + 1)) {
+            auto refill = [&](uint32_t stage, uint32_t bar) {
+                if (vfill < total_tiles) load_tile(fill, stage, bar);
+            };
+            if (tile < c.full_tiles)
+                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, c, k, rot, tile, refill,
+                                                                         local_bucket, scale_writer);
+            else
+                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, c, k, rot, tile, refill,
+                                                                          local_bucket, scale_writer);
+            vfill += stride;
+            if (vfill < total_tiles) advance(fill, stride);
+        }
+        while (tile >= a.ntiles) { tile -= a.ntiles; ++w; }     // into the next worker (if the walk goes on)
     }
     if (!ok) {                         // as in the one-worker kernel
         if (t == 0) {
