@@ -633,17 +633,10 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
         for (int w = 0; w < W && aligned; ++w) aligned = aligned16(codes[w] + code_off[j]);
         return aligned;
     };
-    const mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
-        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
-            const cudaError_t err = mqg::launch_server_segments(ptrs, W, bits, tab, first, params,
-                                                                lr, acc_out, stream);
-            if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
-            return MQG_OK;
-        }, own);
-    if (st != MQG_OK) return st;
-    // all long segments together, kMaxServerSegsPerLaunch per launch
+    // the long segments first (they decide how the short ones are handled)
     std::vector<mqg::ServerSegHost> longs;
-    for (int j = 0; j < nseg; ++j) {
+    for (int j = 0; nseg > 0 && seg_off && code_off && j < nseg; ++j) {
+        if (seg_off[j + 1] < seg_off[j]) break;          // a bad table: for_each_chunk below reports it
         if (!own(j)) continue;
         mqg::ServerSegHost h;
         h.n = seg_off[j + 1] - seg_off[j];
@@ -652,11 +645,28 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
         h.scale_idx = (uint32_t)j;
         longs.push_back(h);
     }
+    // The other segments: table-driven launches - except that ONE table of short segments rides along
+    // with the (first) launch of the long ones, so that a typical layered step is a single launch.
+    std::vector<std::pair<mqg::SegmentTable, int>> short_tabs;
+    const mqg_status st = for_each_chunk(nseg, seg_off, code_off, bits,
+        [&](const mqg::SegmentTable& tab, int first) -> mqg_status {
+            if (tab.tile_start[tab.nseg] != 0) short_tabs.emplace_back(tab, first);
+            return MQG_OK;
+        }, own);
+    if (st != MQG_OK) return st;
+    const bool fold = !longs.empty() && !short_tabs.empty();
+    for (size_t i = fold ? 1 : 0; i < short_tabs.size(); ++i) {
+        const cudaError_t err = mqg::launch_server_segments(ptrs, W, bits, short_tabs[i].first, short_tabs[i].second,
+                                                            params, lr, acc_out, stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
+    }
     for (size_t i = 0; i < longs.size(); i += (size_t)mqg::kMaxServerSegsPerLaunch) {
         const size_t cnt = longs.size() - i < (size_t)mqg::kMaxServerSegsPerLaunch ? longs.size() - i
                                                                                    : (size_t)mqg::kMaxServerSegsPerLaunch;
-        const cudaError_t err = mqg::launch_server_tma_segments(ptrs, W, bits, longs.data() + i, (int)cnt, params, lr,
-                                                                stream);
+        const bool with_short = fold && i == 0;
+        const cudaError_t err = mqg::launch_server_tma_segments(
+            ptrs, W, bits, longs.data() + i, (int)cnt, with_short ? &short_tabs[0].first : nullptr,
+            with_short ? short_tabs[0].second : 0, params, lr, stream);
         if (err != cudaSuccess) return cuda_fail("mqg_server_step_segments", err);
     }
     return MQG_OK;

@@ -142,8 +142,11 @@ struct ServerSegHost {
 };
 constexpr int kMaxServerSegsPerLaunch = 16;
 bool server_tma_segment_applies(uint64_t len);
+// short_tab (may be null): the table of the step's other segments, updated by the same launch with plain
+// loads; short_first = index of the table's first segment in the scale arrays.
 cudaError_t launch_server_tma_segments(const WorkerPtrs& ptrs, int W, int bits, const ServerSegHost* segs, int nseg,
-                                       float* params, float lr, cudaStream_t stream);
+                                       const SegmentTable* short_tab, int short_first, float* params, float lr,
+                                       cudaStream_t stream);
 
 cudaError_t launch_server_segments(const WorkerPtrs& ptrs, int W, int bits, const SegmentTable& tab,
                                    int scale_base, float* params, float lr, float* acc,

@@ -19,8 +19,7 @@
 
 #include <atomic>
 
-#include "mqg_common.cuh"
-#include "mqg_internal.h"
+#include "mqg_segments.cuh"
 #include "mqg_tma.cuh"
 
 namespace mqg {
@@ -526,13 +525,78 @@ server_tma_kernel(const __grid_constant__ CUtensorMap map_full, const __grid_con
     server_tma_body<BITS, MODE, RANGE, false>(&map_full, a, nullptr, timeouts);
 }
 
-// Several long segments of a per-layer step (fused update only).
+// The short segments of a per-layer step (those that are not entries of the segment table): their
+// tiles come from the table-driven layout of mqg_segments.cuh, cut into pieces of 32 rows, one per warp
+// turn.  A lane owns a row: plain loads of its code words, four workers requested at a time, and of its
+// 32 parameters.  A few per cent of a layered gradient; folded into the launch of the long segments so
+// that the step is one launch.
+struct ServerShortSegs {
+    SegmentTable tab;
+    int scale_first;             // index of the table's first segment in every worker's scale array
+    uint32_t pieces;             // 8 x tiles of the table
+};
+
+template <int BITS>
+__device__ __noinline__ void server_short_piece(const ServerTmaArgs& a, const ServerShortSegs& ss, uint32_t piece,
+                                                uint32_t lane)
+{
+    const TileGeom g = locate_tile<BITS>(ss.tab, piece >> 3);
+    const uint32_t r = (piece & 7u) * 32u + lane;
+    if (r >= (uint32_t)g.rows) return;
+    const uint64_t e0 = g.elem0 + 32ull * r;
+    const uint64_t left = g.valid - 32ull * r;            // elements from this row to the segment's end
+    const uint64_t word0 = g.word0 + (uint64_t)r * BITS;
+    const uint64_t scale_idx = (uint64_t)ss.scale_first + g.seg;
+    float2 v2[16];
+#pragma unroll
+    for (int p = 0; p < 16; ++p) v2[p] = make_float2(0.0f, 0.0f);
+    constexpr int kBatch = 4;
+    for (int w0 = 0; w0 < a.W; w0 += kBatch) {
+        uint32_t cw[kBatch][BITS];
+        float sc[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int wk = min(w0 + i, a.W - 1);          // a worker past the last one repeats it (not summed)
+#pragma unroll
+            for (int k = 0; k < BITS; ++k)
+                cw[i][k] = (word0 + k < g.words_end) ? __ldg(a.ptrs.codes[wk] + word0 + k) : 0u;
+            sc[i] = __ldg(a.ptrs.scales[wk] + scale_idx);
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i)
+            if (w0 + i < a.W) add_decoded_row<BITS>(cw[i], widen(decode_scale<BITS>(sc[i])), v2);
+    }
+    float* p = a.params + e0;
+    if (left >= 32 && (reinterpret_cast<uintptr_t>(p) & 15u) == 0) {
+        const float2 nlr = make_float2(a.neg_lr, a.neg_lr);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float4 q = reinterpret_cast<const float4*>(p)[c];
+            const float2 lo = __ffma2_rn(nlr, v2[2 * c], make_float2(q.x, q.y));
+            const float2 hi = __ffma2_rn(nlr, v2[2 * c + 1], make_float2(q.z, q.w));
+            reinterpret_cast<float4*>(p)[c] = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+    } else {
+        float v[32];
+        floats_from_pairs(v2, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if ((uint64_t)j < left) p[j] = __fmaf_rn(a.neg_lr, v[j], p[j]);
+    }
+}
+
+// Several long segments of a per-layer step (fused update only), then the step's short segments.
 template <int BITS>
 __global__ void __launch_bounds__(kSrvThreads, server_min_ctas<BITS>())
-server_tma_segments_kernel(const __grid_constant__ ServerSegTable segs, const __grid_constant__ ServerTmaArgs a,
-                           unsigned int* __restrict__ timeouts)
+server_tma_segments_kernel(const __grid_constant__ ServerSegTable segs, const __grid_constant__ ServerShortSegs ss,
+                           const __grid_constant__ ServerTmaArgs a, unsigned int* __restrict__ timeouts)
 {
     server_tma_body<BITS, 1, false, true>(nullptr, a, &segs, timeouts);
+    const uint32_t wid = __shfl_sync(0xFFFFFFFFu, threadIdx.x >> 5, 0);
+    const uint32_t nwarps = gridDim.x * kSrvWarps;
+    // the warps that finished their share of the long segments first are the last ones of the grid
+    for (uint32_t piece = nwarps - 1 - (blockIdx.x * kSrvWarps + wid); piece < ss.pieces; piece += nwarps)
+        server_short_piece<BITS>(a, ss, piece, threadIdx.x & 31u);
 }
 
 template <int BITS, int MODE, bool RANGE>
@@ -934,8 +998,8 @@ cudaError_t launch_requantize_warp(const WorkerPtrs& ptrs, int W, int bits, uint
 
 // ---- several long segments of a per-layer step in one launch --------------------------------------
 template <int BITS>
-static cudaError_t launch_server_segs_inst(const ServerSegTable& tab, const ServerTmaArgs& a, unsigned int* timeouts,
-                                           cudaStream_t stream)
+static cudaError_t launch_server_segs_inst(const ServerSegTable& tab, const ServerShortSegs& ss, const ServerTmaArgs& a,
+                                           unsigned int* timeouts, cudaStream_t stream)
 {
     auto kernel = server_tma_segments_kernel<BITS>;
     constexpr size_t kSmemBytes = sizeof(ServerSmem<BITS>) + 1024;   // + slack to round the base up
@@ -959,15 +1023,25 @@ static cudaError_t launch_server_segs_inst(const ServerSegTable& tab, const Serv
     uint64_t grid = (uint64_t)cap;
     const uint64_t max_warps = (a.ntiles + 3) / 4;
     if (grid * kSrvWarps > max_warps) grid = (max_warps + kSrvWarps - 1) / kSrvWarps;
-    return launch_pdl_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, tab, a, timeouts);
+    return launch_pdl_smem(kernel, (unsigned)grid, kSrvThreads, kSmemBytes, stream, tab, ss, a, timeouts);
 }
 
 bool server_tma_segment_applies(uint64_t len) { return server_tma_applies(len, len); }
 
 cudaError_t launch_server_tma_segments(const WorkerPtrs& ptrs, int W, int bits, const ServerSegHost* segs, int nseg,
-                                       float* params, float lr, cudaStream_t stream)
+                                       const SegmentTable* short_tab, int short_first, float* params, float lr,
+                                       cudaStream_t stream)
 {
     if (nseg < 1 || nseg > kMaxSrvSegs) return cudaErrorInvalidValue;
+    ServerShortSegs ss;
+    memset(&ss, 0, sizeof(ss));
+    if (short_tab != nullptr) {
+        const uint64_t pieces = 8ull * short_tab->tile_start[short_tab->nseg];
+        if (pieces > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+        ss.tab = *short_tab;
+        ss.scale_first = short_first;
+        ss.pieces = (uint32_t)pieces;
+    }
     ServerSegTable tab;
     memset(&tab, 0, sizeof(tab));
     tab.nseg = nseg;
@@ -1008,14 +1082,14 @@ cudaError_t launch_server_tma_segments(const WorkerPtrs& ptrs, int W, int bits, 
     unsigned int* timeouts = wait_timeout_counter();
     if (timeouts == nullptr) return cudaErrorNotSupported;
     switch (bits) {
-        case 1: return launch_server_segs_inst<1>(tab, a, timeouts, stream);
-        case 2: return launch_server_segs_inst<2>(tab, a, timeouts, stream);
-        case 3: return launch_server_segs_inst<3>(tab, a, timeouts, stream);
-        case 4: return launch_server_segs_inst<4>(tab, a, timeouts, stream);
-        case 5: return launch_server_segs_inst<5>(tab, a, timeouts, stream);
-        case 6: return launch_server_segs_inst<6>(tab, a, timeouts, stream);
-        case 7: return launch_server_segs_inst<7>(tab, a, timeouts, stream);
-        case 8: return launch_server_segs_inst<8>(tab, a, timeouts, stream);
+        case 1: return launch_server_segs_inst<1>(tab, ss, a, timeouts, stream);
+        case 2: return launch_server_segs_inst<2>(tab, ss, a, timeouts, stream);
+        case 3: return launch_server_segs_inst<3>(tab, ss, a, timeouts, stream);
+        case 4: return launch_server_segs_inst<4>(tab, ss, a, timeouts, stream);
+        case 5: return launch_server_segs_inst<5>(tab, ss, a, timeouts, stream);
+        case 6: return launch_server_segs_inst<6>(tab, ss, a, timeouts, stream);
+        case 7: return launch_server_segs_inst<7>(tab, ss, a, timeouts, stream);
+        case 8: return launch_server_segs_inst<8>(tab, ss, a, timeouts, stream);
     }
     return cudaErrorInvalidValue;
 }
