@@ -322,6 +322,29 @@ def test_segments_long_segments_take_their_own_launches(bits):
     assert mqg.mqg_device_timeouts() == 0
 
 
+def test_segments_more_long_segments_than_one_server_launch_holds():
+    """18 long segments (16 per launch of the segment server kernel) between short ones, ragged lengths."""
+    bits, W = 5, 2
+    sizes = []
+    for j in range(18):                  # multiples of 128 elements keep every segment's buffers 16-byte aligned
+        sizes += [(1 << 20) + 128 * j, 128 * (1 + j % 3)]
+    sizes[-2] += 7                       # the last long segment ends with a ragged row
+    sizes[-1] = 45
+    seg, coff = _segments(sizes, bits)
+    n = int(seg[-1])
+    xs = [wl.layered(sizes, config=3, worker=w) for w in range(W)]
+    refs = [O.quantize_segments(x, seg, coff, bits, seed=6, worker=w) for w, x in enumerate(xs)]
+    codes, scales = [r[0] for r in refs], [r[1] for r in refs]
+    p0 = wl.params(n, 0.05, config=3)
+    p_ref, _ = O.server_step_segments(codes, scales, bits, seg, coff, p0.copy(), 0.05)
+    p = Guarded(n, torch.float32, fill=p0)
+    mqg.mqg_server_step_segments([to_dev(c.view(np.int32)) for c in codes], [to_dev(s) for s in scales],
+                                 W, bits, seg, coff, p.view, 0.05)
+    torch.cuda.synchronize()
+    p.check_guards()
+    assert bits_equal(p.numpy(np.float32), p_ref) == 0
+
+
 def test_segments_more_than_one_launch_chunk():
     rng = np.random.default_rng(0)
     sizes = [int(v) for v in rng.integers(0, 600, 150)]
@@ -347,7 +370,7 @@ def test_segments_more_than_one_launch_chunk():
                                         # buckets; worker counts that do not fill a code stage; 32 workers)
                                         ((1 << 17) + 64, 2048, 8), ((1 << 17) + 5 * 1024, 4096, 3), (99_968, 1024, 5),
                                         (32_768 + 64, 256, 8), (16_384 + 32, 32, 2), (22_400, 64, 4),
-                                        (1 << 15, 2048, 32), ((1 << 16) + 2048 + 32, 2048, 9)])
+                                        (1 << 15, 2048, 32), ((1 << 16) + 2048 + 32, 2048, 9), (1 << 16, 2048, 1)])
 def test_server_requantize(bits, n, bucket, W):
     xs = [wl.normal(n, 2e-3, config=41, worker=w) for w in range(W)]
     if n >= bucket:
