@@ -275,6 +275,35 @@ __device__ __forceinline__ void encode_pack_row(const float (&x)[32], const Enco
     }
 }
 
+// The same with the packed fp32x2 instructions of sm_100: two elements per instruction, each lane rounded
+// exactly as the scalar instruction would.  |T| is not taken: a T rounded slightly below zero gives a
+// negative difference in (-2^16, 0) either way, and the ceiling of that is code 0.
+template <int BITS>
+__device__ __forceinline__ void encode_pack_row_packed(const float (&x)[32], const EncodeScale& e,
+                                                       const uint32_t (&h)[16], uint32_t (&w)[BITS])
+{
+    const float2 inv = make_float2(e.inv16, e.inv16), half = make_float2(e.half_l16, e.half_l16);
+    const float2 neg1 = make_float2(-1.0f, -1.0f), c = make_float2(8388607.5f, 8388607.5f);
+    const float2 r16 = make_float2(1.0f / 65536.0f, 1.0f / 65536.0f), magic = make_float2(12582912.0f, 12582912.0f);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+        const float2 hf = make_float2(draw_lo(h[p]), draw_hi(h[p]));
+        const float2 T = __ffma2_rn(make_float2(x[2 * p], x[2 * p + 1]), inv, half);
+        const float2 nhh = __ffma2_rn(hf, neg1, c);             // -(h + 1/2), exact
+        const float2 d = __fadd2_ru(T, nhh);
+        const float2 ww = __ffma2_ru(d, r16, magic);
+        const uint32_t cc[2] = {__float_as_uint(ww.x), __float_as_uint(ww.y)};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int j = 2 * p + q;
+            const int o = j * BITS, wi = o >> 5, sh = o & 31;
+            if (sh == 0) w[wi] = cc[q] - pack_bias<BITS>(wi);
+            else w[wi] = w[wi] + (cc[q] << sh);
+            if (sh + BITS > 32) w[wi + 1] = (cc[q] >> (32 - sh)) - pack_bias<BITS>(wi + 1);
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------
 // Codec variant: (min, max) range with nearest rounding.  Per bucket lo = min x, hi = max x
 // (a zero of either sign stored as +0), r = fl(hi - lo); code = min(L, floor(fma(fl(x - lo),

@@ -214,7 +214,11 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     if constexpr (!NORM && !kEarlyDraw)
         draw_row_blocks_head(wv.blk0_lo + 4u * row, wv.head, c.rk, h);
     uint32_t w[BITS];
-    encode_pack_row<BITS>(x, es, h, w);
+    // one and two bits: the encode's arithmetic with the packed fp32x2 instructions (per 100 MB gradient in the
+    // batched launch 16.6 against 17.2 us at K = 1, 17.0 against 17.3 us at K = 2; no gain at K = 3, a loss from
+    // K = 4 on, where the constant pairs and the early draws compete for registers: 18.6 against 17.6 us at K = 4)
+    if constexpr (BITS <= 2) encode_pack_row_packed<BITS>(x, es, h, w);
+    else encode_pack_row<BITS>(x, es, h, w);
     const uint64_t word0 = (uint64_t)row * BITS;
     if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
         store_row_words<BITS>(wv.codes, word0, w);
