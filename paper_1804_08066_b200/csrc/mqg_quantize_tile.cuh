@@ -216,8 +216,11 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     uint32_t w[BITS];
     // one and two bits: the encode's arithmetic with the packed fp32x2 instructions (per 100 MB gradient in the
     // batched launch 16.6 against 17.2 us at K = 1, 17.0 against 17.3 us at K = 2; no gain at K = 3, a loss from
-    // K = 4 on, where the constant pairs and the early draws compete for registers: 18.6 against 17.6 us at K = 4)
-    if constexpr (BITS <= 2) encode_pack_row_packed<BITS>(x, es, h, w);
+    // K = 4 on, where the constant pairs and the early draws compete for registers: 18.6 against 17.6 us at K = 4).
+    // bf16 input at every width: per 50 MB gradient (bucket 4096) 16.4 against 17.8 us at K = 3, 16.4 against
+    // 17.7 at K = 4, 17.1 .. 17.3 against 18.2 .. 18.5 at K = 5 .. 7, 16.7 against 17.8 at K = 8.
+    constexpr bool kPackedEncode = DTYPE == 1 || BITS <= 2;
+    if constexpr (kPackedEncode) encode_pack_row_packed<BITS>(x, es, h, w);
     else encode_pack_row<BITS>(x, es, h, w);
     const uint64_t word0 = (uint64_t)row * BITS;
     if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
