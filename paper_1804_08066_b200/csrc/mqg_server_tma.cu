@@ -904,7 +904,10 @@ requantize_warp_kernel(const __grid_constant__ RequantWarpArgs ra)
             uint32_t h[16];
             draw_row_blocks_head(4u * row, ra.head, ra.rk, h);     // the downlink draws from position 0
             uint32_t w[BITS];
-            encode_pack_row<BITS>(x, es, h, w);
+            // (the encode's arithmetic in packed fp32x2 instructions: 0.5 to 1 us per launch at every width;
+            // a fifth resident CTA, which 95 registers would allow, changes nothing: the kernel waits on
+            // its arithmetic pipes, not on latency)
+            encode_pack_row_packed<BITS>(x, es, h, w);
             store_row_words<BITS>(ra.codes_out, (uint64_t)row * BITS, w);
         }
         if (have_next) store_tile_scales<BITS, false>(a, table, lane, wide, s_next);
