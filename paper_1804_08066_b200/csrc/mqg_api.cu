@@ -442,7 +442,7 @@ mqg_status mqg_quantize_segments_workers(const void* const* grads, int W, int ns
         for (int w = 0; w < W; ++w)
             if (!mqg::quantize_given_scale_applies(static_cast<const char*>(grads[w]) + seg_off[j] * esz,
                                                    seg_off[j + 1] - seg_off[j], codes[w] + code_off[j],
-                                                   elem_offset + seg_off[j]))
+                                                   elem_offset + seg_off[j], mqg::kEntrySegmentElems))
                 return false;
         return true;
     };
@@ -625,7 +625,7 @@ mqg_status mqg_server_step_segments(const uint32_t* const* codes, const float* c
     // A long segment is a gradient with a single bucket: the long segments whose buffers are aligned for
     // bulk copies go to the TMA-fed server kernel together, in one launch; all other segments share
     // the table-driven launch.  The results are the same bit for bit either way.
-    constexpr uint64_t kOwnLaunchElems = 1ull << 20;
+    constexpr uint64_t kOwnLaunchElems = mqg::kEntrySegmentElems;
     auto own = [&](int j) {
         const uint64_t len = seg_off[j + 1] - seg_off[j];
         if (acc_out || len < kOwnLaunchElems || !mqg::server_tma_applies(len, len)) return false;

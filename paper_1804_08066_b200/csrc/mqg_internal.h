@@ -86,7 +86,15 @@ cudaError_t launch_segments_absmax(const void* grad, const SegmentTable& tab, fl
 cudaError_t launch_segments_encode(const void* grad, const SegmentTable& tab, int bits, uint64_t seed,
                                    uint32_t* codes, float* scales_base, int dtype, uint32_t worker,
                                    uint32_t step, uint64_t elem_offset, cudaStream_t stream);
-bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset);
+// Shortest segment that gets a launch of its own on the bulk-copy kernels (one-worker per-layer calls), and
+// shortest segment that becomes one entry of a launch shared by many segments (the all-workers quantizer,
+// the per-layer server step): 8 tiles of 128 rows.  Shorter segments go through the table-driven code.
+// (Entries from 2^15 instead of 2^20 elements on the AlexNet-shaped gradient, W = 8: the five convolution
+// tensors join the three large ones; quantize call 620 against 631 us, server step 137 against 140 us at K = 4.)
+constexpr uint64_t kOwnLaunchSegmentElems = 1ull << 20;
+constexpr uint64_t kEntrySegmentElems = 1ull << 15;
+bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset,
+                                  uint64_t min_elems = kOwnLaunchSegmentElems);
 cudaError_t launch_quantize_given_scale(const void* grad, uint64_t n, int bits, uint64_t seed, uint32_t* codes,
                                         float* scale, int dtype, uint32_t worker, uint32_t step,
                                         uint64_t elem_offset, cudaStream_t stream);
@@ -102,7 +110,7 @@ struct SegEntryHost {
     uint64_t elem_offset;    // flat position of its first element (for the draws)
     uint32_t worker;         // worker id of the draws
 };
-constexpr int kMaxSegEntriesPerLaunch = 32;
+constexpr int kMaxSegEntriesPerLaunch = 64;
 cudaError_t launch_zero_scales(float* const* scales, int W, int nseg, cudaStream_t stream);
 cudaError_t launch_absmax_workers(const void* const* grads, float* const* scales, int first, int W,
                                   const SegmentTable& tab, int dtype, cudaStream_t stream);

@@ -723,9 +723,10 @@ cudaError_t launch_quantize_norm_fused(const void* grad, uint64_t n, int bits, u
 }
 
 // ---- encode against a given scale on the TMA kernel: one long segment (= one bucket) per launch ----
-bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset)
+bool quantize_given_scale_applies(const void* grad, uint64_t n, const uint32_t* codes, uint64_t elem_offset,
+                                  uint64_t min_elems)
 {
-    return n >= (1ull << 20) && n / 32 <= 0x7FFFFFFFull && (elem_offset & 7u) == 0 &&
+    return n >= min_elems && n / 32 <= 0x7FFFFFFFull && (elem_offset & 7u) == 0 &&
            blocks_share_high_half(n, elem_offset) &&
            (reinterpret_cast<uintptr_t>(grad) & 15u) == 0 && (reinterpret_cast<uintptr_t>(codes) & 15u) == 0;
 }

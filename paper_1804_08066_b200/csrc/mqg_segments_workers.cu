@@ -18,7 +18,7 @@
 
 namespace mqg {
 
-constexpr int kMaxSegEntries = 32;        // (worker, long segment) pairs per launch
+constexpr int kMaxSegEntries = kMaxSegEntriesPerLaunch;        // (worker, long segment) pairs per launch
 
 struct SegEntry {
     const void* grad;        // the segment's first element (for its ragged last row)

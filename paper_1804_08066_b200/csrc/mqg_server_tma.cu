@@ -36,6 +36,14 @@ constexpr int kCodeDepth = 2;                     // code stages per warp
 template <int BITS>
 struct ServerGroup { static constexpr int value = BITS <= 4 ? 8 : 4; };
 
+// Barrier ID (1 .. 15; 0 is the one of __syncthreads) among `threads` threads of a CTA (a multiple of 32:
+// whole warps); every thread that takes part names the same count.
+template <int ID>
+__device__ __forceinline__ void named_barrier(uint32_t threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "r"(threads) : "memory");
+}
+
 struct ServerTmaArgs {
     WorkerPtrs ptrs;
     float* params;
@@ -306,13 +314,22 @@ __device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, con
     __syncwarp();
     grid_dependency_wait();            // nothing above touches global memory
 
-    // this warp's tiles: [t_begin, t_begin + ntiles), the grid's tiles split evenly; the warps of the
-    // first CTAs take the odd tiles (they start first; spreading the odd tiles evenly over the grid
-    // measured 2 us slower per launch)
+    // This warp's tiles: gwarp, gwarp + nwarps, gwarp + 2 nwarps, ...  At any moment the grid then works
+    // on one window of consecutive tiles, and the four warps of a CTA on four consecutive ones: their
+    // requests for a worker's code words (32 K bytes per tile) fall into the same DRAM pages at about the
+    // same time.  Against a contiguous range of tiles per warp, per launch at eight workers: 37.5 against
+    // 39.7 us at one bit, 44.5 against 47.6 at three, 61.0 against 63.0 at eight (n = 25 M); 89 against 94,
+    // 115 against 123, 143 against 147 us at n = 61 M.
     const uint32_t gwarp = blockIdx.x * kSrvWarps + wid, nwarps = gridDim.x * kSrvWarps;
     const uint32_t base = a.ntiles / nwarps, extra = a.ntiles % nwarps;
-    const uint32_t t_begin = gwarp * base + min(gwarp, extra);
+    const uint32_t t_begin = gwarp, t_step = nwarps;
     const uint32_t ntiles = base + (gwarp < extra ? 1u : 0u);
+    // Three and four bits: the warps of a CTA start every tile together (a CTA barrier per tile, for the
+    // `base` tiles that every warp of the grid has), which keeps those requests together for the whole
+    // launch: 106 against 116 us at three bits, 121 against 127 us at four (n = 61 M; 44.3 and 46.9 against
+    // 44.3 and 48.0 us at n = 25 M); no gain at one and two bits, a loss of 1 to 2 % from five bits on.
+    constexpr bool kCtaSync = BITS == 3 || BITS == 4;
+    const uint32_t sync_tiles = base;
     const uint32_t last_row = a.nrows_full - 1;    // nrows_full >= 1 on this path (not used by SEGS)
     uint32_t cur_e = 0, next_e = 0, fill_e = 0;    // SEGS: segment cursors of the tile in work, the next
                                                    // tile (its scales) and the tile whose codes are fetched
@@ -343,7 +360,7 @@ __device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, con
         for (uint32_t u2 = 0; u2 < (uint32_t)kCodeDepth; ++u2) {
             if (u2 < nunits)
                 fill_code_stage<BITS>(a, code_base + u2 * kCodeStageBytes,
-                                      locate_srv_tile<SEGS>(map_full, a, segs, t_begin + u2 / groups, fill_e),
+                                      locate_srv_tile<SEGS>(map_full, a, segs, t_begin + (u2 / groups) * t_step, fill_e),
                                       (int)(u2 % groups) * kGroup, lane_off);
             cp_async_commit();
         }
@@ -354,14 +371,17 @@ __device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, con
 
 #pragma unroll 1
     for (; k < ntiles; ++k) {
+        if constexpr (kCtaSync) {
+            if (k < sync_tiles) named_barrier<1>(kSrvThreads);
+        }
         const uint32_t parity = k & 1;
-        const TileLoc loc = locate_srv_tile<SEGS>(map_full, a, segs, t_begin + k, cur_e);
+        const TileLoc loc = locate_srv_tile<SEGS>(map_full, a, segs, t_begin + k * t_step, cur_e);
         const uint32_t row0 = loc.row0;
         const bool have_next = k + 1 < ntiles;
         float2 s_next[2];
         TileLoc loc_next = loc;
         if (have_next) {
-            loc_next = locate_srv_tile<SEGS>(map_full, a, segs, t_begin + k + 1, next_e);
+            loc_next = locate_srv_tile<SEGS>(map_full, a, segs, t_begin + (k + 1) * t_step, next_e);
             load_tile_scales<RANGE, SEGS>(a, loc_next, lane, wide, s_next);
         }
 
@@ -419,12 +439,18 @@ __device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, con
                     if (!a.arm_only) tma_load_2d(smem_u32(stage), loc.map, 0, (int)row0, bar);
                 }
             };
-            if (g0 + kGroup <= a.W) {              // a whole stage: straight-line code
+            static_assert(kIssueAt == 4 && kGroup % 4 == 0, "the parameter load is issued between blocks of four workers");
+            if (g0 + kGroup <= a.W) {              // a whole stage: blocks of four workers in straight-line code
+#pragma unroll 1
+                for (int i0 = 0; i0 < kGroup; i0 += 4) {
+                    // (the positions a whole stage can hold issue_at at: worker 4 when W >= 5, else the
+                    // stage's last worker when W == group size)
+                    if (MODE == 1 && g0 + i0 == issue_at) load_params();
 #pragma unroll
-                for (int i = 0; i < kGroup; ++i) {
-                    // (the two positions a whole stage can hold issue_at at: W >= 5, and W == group size)
-                    if (MODE == 1 && (i == kIssueAt % kGroup || i == kGroup - 1) && g0 + i == issue_at) load_params();
-                    decode_worker(i);
+                    for (int i = 0; i < 4; ++i) {
+                        if (MODE == 1 && i == 3 && i0 + i == kGroup - 1 && g0 + i0 + i == issue_at) load_params();
+                        decode_worker(i0 + i);
+                    }
                 }
             } else {
 #pragma unroll 1
@@ -436,7 +462,7 @@ __device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, con
             __syncwarp();                          // every lane has read the stage: refill it
             if (u + kCodeDepth < nunits)
                 fill_code_stage<BITS>(a, cstage_addr,
-                                      locate_srv_tile<SEGS>(map_full, a, segs, t_begin + fill_tile, fill_e),
+                                      locate_srv_tile<SEGS>(map_full, a, segs, t_begin + fill_tile * t_step, fill_e),
                                       (int)fill_group * kGroup, lane_off);
             cp_async_commit();
             if (++fill_group == groups) { fill_group = 0; ++fill_tile; }
@@ -486,6 +512,10 @@ __device__ __forceinline__ void server_tma_body(const CUtensorMap* map_full, con
                 if (!a.arm_only) tma_load_2d(smem_u32(stage), loc_next.map, 0, (int)loc_next.row0, bar);
             }
         }
+    }
+    if constexpr (kCtaSync) {
+        if (failed)                     // a warp that gave up still arrives at the barriers the others expect
+            for (uint32_t kk = k + 1; kk < sync_tiles; ++kk) named_barrier<1>(kSrvThreads);
     }
     cp_async_wait_group<0>();                                  // no code copy outlives the warp
     if (lane == 0) {
@@ -759,12 +789,6 @@ struct RequantSmem {
     uint32_t bmax[2][kSrvWarps];                  // tile maxima, double-buffered by the parity of the turn
 };
 
-template <int ID>
-__device__ __forceinline__ void named_barrier(uint32_t threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"n"(ID), "r"(threads) : "memory");
-}
-
 template <int BITS>
 __global__ void __launch_bounds__(kSrvThreads, 4)
 requantize_warp_kernel(const __grid_constant__ RequantWarpArgs ra)
@@ -782,9 +806,9 @@ requantize_warp_kernel(const __grid_constant__ RequantWarpArgs ra)
     const uint32_t code_base = smem_u32(&sm.code[wid][0][0][0]);
     grid_dependency_wait();            // nothing above touches global memory
 
-    // this CTA's tiles of 128 rows: [ct_begin, ct_begin + nct); warp w takes rows 32 w .. 32 w + 31 of each
+    // this CTA's tiles of 128 rows: blockIdx.x, blockIdx.x + gridDim.x, ... (the grid works on one window of
+    // consecutive tiles at a time, as in the server kernel); warp w takes rows 32 w .. 32 w + 31 of each
     const uint32_t base = ra.nct / gridDim.x, extra = ra.nct % gridDim.x;
-    const uint32_t ct_begin = blockIdx.x * base + min(blockIdx.x, extra);
     const uint32_t nct = base + (blockIdx.x < extra ? 1u : 0u);
     const uint32_t groups = ((uint32_t)a.W + kGroup - 1) / kGroup;      // code stages per tile
     const uint32_t nunits = nct * groups;
@@ -795,7 +819,7 @@ requantize_warp_kernel(const __grid_constant__ RequantWarpArgs ra)
     auto tile_loc = [&](uint32_t kk) {
         TileLoc t;
         t.map = nullptr;
-        t.row0 = ((ct_begin + kk) * kSrvWarps + wid) * kSrvTileRows;
+        t.row0 = ((blockIdx.x + kk * gridDim.x) * kSrvWarps + wid) * kSrvTileRows;
         t.nrows_full = a.nrows_full;
         t.scale_idx = 0;
         t.code_word0 = 0;

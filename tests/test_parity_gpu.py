@@ -323,11 +323,12 @@ def test_segments_long_segments_take_their_own_launches(bits):
 
 
 def test_segments_more_long_segments_than_one_server_launch_holds():
-    """18 long segments (16 per launch of the segment server kernel) between short ones, ragged lengths."""
+    """18 long segments (16 per launch of the segment server kernel; a segment is long from 32,768 elements
+    on) between short ones, ragged lengths."""
     bits, W = 5, 2
     sizes = []
     for j in range(18):                  # multiples of 128 elements keep every segment's buffers 16-byte aligned
-        sizes += [(1 << 20) + 128 * j, 128 * (1 + j % 3)]
+        sizes += [((1 << 20) if j % 2 == 0 else (1 << 15)) + 128 * j, 128 * (1 + j % 3)]
     sizes[-2] += 7                       # the last long segment ends with a ragged row
     sizes[-1] = 45
     seg, coff = _segments(sizes, bits)

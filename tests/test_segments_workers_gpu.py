@@ -2,7 +2,7 @@
 launches for all of them) against the CPU checker, worker by worker and bit for bit, with guard
 words around every output.  Covers short segments only, long segments that become entries of the
 bulk-copy part (ragged lengths, a flushed one), long segments that do not qualify (odd word
-offset), more than 32 (worker, long segment) pairs and more than 64 segments (several launches),
+offset), more than 64 (worker, long segment) pairs and more than 64 segments (several launches),
 bf16 input, worker ids and offsets, and the AlexNet-shaped and Section 4.1 layouts."""
 import numpy as np
 import pytest
@@ -79,10 +79,11 @@ def test_long_and_short_segments(bits):
 
 
 def test_more_pairs_than_one_launch_holds_and_more_segments_than_one_table():
-    """12 workers x 3 long segments = 36 (worker, long segment) pairs (32 per launch) and 150 short
-    segments (64 per table)."""
+    """12 workers x 6 long segments = 72 (worker, long segment) pairs (64 per launch; a segment is an
+    entry from 32,768 elements on) and 150 short segments (64 per table)."""
     rng = np.random.default_rng(1)
-    sizes = [1 << 20, 1 << 20, (1 << 20) + 32] + [int(v) for v in rng.integers(0, 600, 150)]
+    sizes = [1 << 20, 1 << 15, (1 << 20) + 32, (1 << 15) + 4096 + 7, 1 << 16, 40_000 - 32] + \
+        [int(v) for v in rng.integers(0, 600, 150)]
     bits = 5
     seg, coff = _segments(sizes, bits)
     xs = [wl.layered(sizes, config=31, worker=w) for w in range(12)]
