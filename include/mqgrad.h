@@ -274,8 +274,9 @@ mqg_status mqg_quantize_segments_l2_static(const void* grad, int nseg, const uin
  *   codes     [out] code_off[nseg] words;  scales [out] nseg floats
  * Element i of segment j draws with position elem_offset + seg_off[j] + i.  Empty segments get
  * scale 0.  The gradient is read twice (max pass, encode pass).
- * Performance note: a segment of 2^20 elements or more is encoded (and, in mqg_server_step_segments,
- * applied) by the bulk-copy kernels when grad + seg_off[j], codes + code_off[j] (every worker's, on
+ * Performance note: a segment of 2^20 elements or more (2^15 or more in mqg_quantize_segments_workers
+ * and mqg_server_step_segments, where such segments share a launch) is encoded (and, in
+ * mqg_server_step_segments, applied) by the bulk-copy kernels when grad + seg_off[j], codes + code_off[j] (every worker's, on
  * the server) and params + seg_off[j] are 16-byte aligned and elem_offset + seg_off[j] is a multiple
  * of 8; otherwise by the table-driven kernels.  The results do not depend on which kernel ran.
  */
