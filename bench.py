@@ -57,8 +57,8 @@ FALLBACK_HBM_GBS = 6650.0
 # elements; server_tma_kernel: n = 2^25, W = 8; both bucket 2048).  DRAM traffic grows in proportion to the
 # elements, so a launch's traffic is the figure times its elements.  Writes are partly still in L2 when a
 # kernel ends, hence less than the algorithmic bytes (4 + K/8 and 8 + W K/8 per element).
-QUANTIZE_DRAM_BYTES_PER_ELEM = {1: 4.0771, 2: 4.1061, 3: 4.141, 4: 4.2012, 5: 4.2161, 6: 4.2546, 7: 4.3087, 8: 4.3646}
-SERVER_DRAM_BYTES_PER_ELEM = {1: 7.2747, 2: 8.3364, 3: 9.4213, 4: 10.4596, 5: 11.6609, 6: 12.7271, 7: 13.795, 8: 14.8942}
+QUANTIZE_DRAM_BYTES_PER_ELEM = {1: 4.0812, 2: 4.1057, 3: 4.1874, 4: 4.2229, 5: 4.2425, 6: 4.2821, 7: 4.3906, 8: 4.3903}
+SERVER_DRAM_BYTES_PER_ELEM = {1: 7.2455, 2: 8.2828, 3: 9.3616, 4: 10.404, 5: 11.6736, 6: 12.7431, 7: 13.8224, 8: 14.858}
 
 
 def measured_hbm_peak():
