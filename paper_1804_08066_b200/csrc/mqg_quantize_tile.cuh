@@ -132,12 +132,13 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     const uint32_t bar = smem_u32(&sh.bar[stg]);
     uint8_t* stage = sh.stage[stg];
 
-    // The row's draws depend on nothing but its number.  From five bits on they are computed before the
-    // tile's data is waited for (measured per 100 MB gradient, batched launch: 17.9 against 18.3 us at
-    // K = 5, 18.5 against 19.0 us at K = 6, 19.3 against 20.5 us at K = 8; the 16 extra live registers cost
-    // the fifth CTA per SM, and below five bits that costs more than the overlap gains: 17.6 against
-    // 17.2 us at K = 1; forcing five CTAs with the early draws, 92 registers, is slower at every width).
-    constexpr bool kEarlyDraw = !NORM && !GIVEN && BITS >= 5;
+    // The row's draws depend on nothing but its number.  From three bits on they are computed before the
+    // tile's data is waited for: 16 more live registers (four CTAs per SM instead of five) against the
+    // overlap of the Philox rounds with the wait.  Measured per 100 MB gradient in the batched launch with the
+    // SM clock at its maximum: 17.0 against 18.0 us at K = 4, 18.3 against 18.6 us at K = 6, 19.7 against
+    // 20.0 us at K = 8; no difference at one and two bits, which keep the fifth CTA.  (In a long run the power
+    // limit sets the clock and both forms take the same time: the instruction count decides there.)
+    constexpr bool kEarlyDraw = !NORM && !GIVEN && BITS >= 3;
     uint32_t h[16];
     if (kEarlyDraw && active) draw_row_blocks_head(wv.blk0_lo + 4u * row, wv.head, c.rk, h);
     bool ok = mbar_try_wait(bar, parity);
@@ -214,14 +215,14 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     if constexpr (!NORM && !kEarlyDraw)
         draw_row_blocks_head(wv.blk0_lo + 4u * row, wv.head, c.rk, h);
     uint32_t w[BITS];
-    // one and two bits: the encode's arithmetic with the packed fp32x2 instructions (per 100 MB gradient in the
-    // batched launch 16.6 against 17.2 us at K = 1, 17.0 against 17.3 us at K = 2; no gain at K = 3, a loss from
-    // K = 4 on, where the constant pairs and the early draws compete for registers: 18.6 against 17.6 us at K = 4).
-    // bf16 input at every width: per 50 MB gradient (bucket 4096) 16.4 against 17.8 us at K = 3, 16.4 against
-    // 17.7 at K = 4, 17.1 .. 17.3 against 18.2 .. 18.5 at K = 5 .. 7, 16.7 against 17.8 at K = 8.
-    constexpr bool kPackedEncode = DTYPE == 1 || BITS <= 2;
-    if constexpr (kPackedEncode) encode_pack_row_packed<BITS>(x, es, h, w);
-    else encode_pack_row<BITS>(x, es, h, w);
+    // The encode's arithmetic runs in packed fp32x2 instructions at every width: 14.3 instead of 17.0 - 17.6
+    // executed instructions per element.  With the SM clock at its maximum this gains only at one and two bits
+    // (16.6 against 17.2 us per 100 MB gradient at K = 1; from K = 4 on the constant pairs compete with the
+    // early draws for registers), but a launch that runs for more than a few tens of milliseconds is held at
+    // the board's power limit, where the clock falls until the power fits and fewer instructions per element
+    // mean less time: 19.6 against 20.5 us at K = 3, 19.4 against 20.4 us at K = 4, 20.5 against 21.2 us at
+    // K = 5, 20.6 against 21.6 us at K = 8 (batched launch, 0.3 s of launches back to back, 1650 - 1720 MHz).
+    encode_pack_row_packed<BITS>(x, es, h, w);
     const uint64_t word0 = (uint64_t)row * BITS;
     if (FULL || (uint64_t)row * 32 + 32 <= a.n) {
         store_row_words<BITS>(wv.codes, word0, w);
