@@ -17,8 +17,10 @@ metric with the gradients starting in pinned host memory and the updated paramet
 back, copies inside the timed region; `roofline` describes the dominant kernel (the quantize
 kernel) and `roofline_server` the fused server kernel, both from events at the phase boundaries
 inside the timed region; `per_bits` lists both kernels for every bit width, each timed on its own
-after the timed region (groups of 8 launches back to back on rotating buffers: median and best
-group; and 20 launches each between its own events); `cpu_baseline` is the scalar CPU
+after the timed region (groups of 8 launches back to back on rotating buffers after a short idle,
+i.e. with the SM clock at its maximum: median and best group; 20 launches each between its own
+events; and `*_sustained`, the same launch after a quarter of a second of itself back to back,
+when the board's power limit has lowered the clock); `cpu_baseline` is the scalar CPU
 checker timed on a bounded sample of the same workload.
 
 --impl reference times the CPU checker alone (rank 0 only).
@@ -57,7 +59,7 @@ FALLBACK_HBM_GBS = 6650.0
 # elements; server_tma_kernel: n = 2^25, W = 8; both bucket 2048).  DRAM traffic grows in proportion to the
 # elements, so a launch's traffic is the figure times its elements.  Writes are partly still in L2 when a
 # kernel ends, hence less than the algorithmic bytes (4 + K/8 and 8 + W K/8 per element).
-QUANTIZE_DRAM_BYTES_PER_ELEM = {1: 4.0812, 2: 4.1057, 3: 4.1874, 4: 4.2229, 5: 4.2425, 6: 4.2821, 7: 4.3906, 8: 4.3903}
+QUANTIZE_DRAM_BYTES_PER_ELEM = {1: 4.0744, 2: 4.1027, 3: 4.151, 4: 4.1934, 5: 4.229, 6: 4.2763, 7: 4.3382, 8: 4.3993}
 SERVER_DRAM_BYTES_PER_ELEM = {1: 7.2455, 2: 8.2828, 3: 9.3616, 4: 10.404, 5: 11.6736, 6: 12.7431, 7: 13.8224, 8: 14.858}
 
 
@@ -400,9 +402,31 @@ def run_ours(args):
     # over REPS groups of the group's time per launch, `us_best` the best group.  `single` figures are
     # SINGLES launches each between its own pair of events (an event after every launch keeps the next
     # one from being set up while it runs, so these are a few microseconds longer).
+    # Power.  A launch sequence that runs for more than a few tens of milliseconds is held at the board's
+    # power limit: the SM clock falls from its maximum to 1650 - 1800 MHz (seen with 5 ms samples; the
+    # limit is often not reported as a reason) and kernels bound by instruction issue slow down with it.
+    # Both regimes are reported: `*_us` after IDLE_S seconds of idle (clock at its maximum, the regime the
+    # copy-rate denominator was measured in), `*_us_sustained` after SUSTAIN_S seconds of the same launch
+    # back to back.
     GROUP, REPS, SINGLES = 8, 5, 20
+    IDLE_S, SUSTAIN_S = 0.4, 0.25
+
+    def time_sustained(launch, est_ms):
+        warm = max(GROUP, int(SUSTAIN_S * 1e3 / max(est_ms, 1e-3)))
+        count = GROUP * REPS
+        for i in range(warm):
+            launch(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(count):
+            launch(warm + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / count
 
     def time_groups(launch):
+        torch.cuda.synchronize()
+        time.sleep(IDLE_S)
         for i in range(2):
             launch(i)
         out, i = [], 2
@@ -428,10 +452,11 @@ def run_ours(args):
         torch.cuda.synchronize()
         return [e0.elapsed_time(e1) for e0, e1 in pairs]
 
-    q_ms, s_ms, q_single, s_single = {}, {}, {}, {}
+    q_ms, s_ms, q_single, s_single, q_sust, s_sust = {}, {}, {}, {}, {}, {}
     for b in ALL_BITS:
         q_ms[b] = time_groups(lambda i: quantize_all(b, i))
         q_single[b] = time_singles(lambda i: quantize_all(b, 100 + i))
+        q_sust[b] = time_sustained(lambda i: quantize_all(b, 200 + i), float(np.median(q_ms[b])))
         # three sets of this width's code buffers, every parameter replica in turn: 2 launches
         # (> 450 MB of traffic) lie between two uses of a code set, 7 between two uses of a replica
         sets = [code_tab[b]]
@@ -447,6 +472,7 @@ def run_ours(args):
 
         s_ms[b] = time_groups(server_rot)
         s_single[b] = time_singles(server_rot)
+        s_sust[b] = time_sustained(server_rot, float(np.median(s_ms[b])))
         del keep, sets
     torch.cuda.synchronize()
 
@@ -484,6 +510,10 @@ def run_ours(args):
             "quantize_frac_of_measured": qb / tq / 1e9 / peak, "quantize_frac_of_8tbs": qb / tq / 1e9 / NOMINAL_HBM_GBS,
             "server_us": ts * 1e6, "server_grad_gbs": 4 * n * W / ts / 1e9, "server_moved_gbs": sb / ts / 1e9,
             "server_frac_of_measured": sb / ts / 1e9 / peak, "server_frac_of_8tbs": sb / ts / 1e9 / NOMINAL_HBM_GBS,
+            "quantize_us_sustained": q_sust[b] / W * 1e3,
+            "quantize_frac_of_measured_sustained": qb / (q_sust[b] / W * 1e-3) / 1e9 / peak,
+            "server_us_sustained": s_sust[b] * 1e3,
+            "server_frac_of_measured_sustained": sb / (s_sust[b] * 1e-3) / 1e9 / peak,
             "quantize_us_best": min(q_ms[b]) / W * 1e3,
             "quantize_us_single_median": float(np.median(q_single[b])) / W * 1e3,
             "quantize_us_single_best": min(q_single[b]) / W * 1e3,
@@ -691,6 +721,9 @@ def run_ours(args):
             "variant_minmax": variant_minmax, "variant_l2": variant_l2,
             "variant_1bit_ef": variant_1bit_ef,
             "per_bits": per_bits,
+            "per_bits_note": "`*_us`: groups of launches after 0.4 s of idle (SM clock at its maximum); "
+                             "`*_us_sustained`: after 0.25 s of the same launch back to back, when the board's "
+                             "power limit has lowered the SM clock (1650-1800 MHz seen)",
         }
         if other_configs is not None:
             line["configs"] = other_configs
@@ -835,10 +868,60 @@ def run_single_kernel(args):
     torch.cuda.synchronize()
     avg = e0.elapsed_time(e1) * 1e-3 / args.launches
     peak, kind = measured_hbm_peak()
-    print(json.dumps({"kernel": args.kernel, "bits": b, "n": n, "workers": W, "bucket": B,
-                      "launches": args.launches, "avg_us": avg * 1e6, "algorithmic_bytes": nbytes,
-                      "avg_gbs": nbytes / avg / 1e9, "frac_of_%s_peak" % kind: nbytes / avg / 1e9 / peak}))
+    line = {"kernel": args.kernel, "bits": b, "n": n, "workers": W, "bucket": B,
+            "launches": args.launches, "avg_us": avg * 1e6, "algorithmic_bytes": nbytes,
+            "avg_gbs": nbytes / avg / 1e9, "frac_of_%s_peak" % kind: nbytes / avg / 1e9 / peak}
+    if args.clock_trace > 0:
+        line["clock_trace"] = clock_trace(torch, stream, launch, avg, args.clock_trace)
+    print(json.dumps(line))
     return 0
+
+
+def clock_trace(torch, stream, launch, est_s, seconds):
+    """The same launch back to back for `seconds` after one second of idle, an event every few launches and
+    the SM clock, the board power and the throttle reasons read through NVML every 5 ms: shows the time per
+    launch following the clock down once the board's power limit acts.  Returns rows of 25 ms."""
+    import pynvml
+    pynvml.nvmlInit()
+    h = pynvml.nvmlDeviceGetHandleByIndex(torch.cuda.current_device())
+    samples, stop = [], threading.Event()
+
+    def sample():
+        while not stop.is_set():
+            samples.append((time.perf_counter(), pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM),
+                            pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0,
+                            int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))))
+            stop.wait(0.005)
+
+    torch.cuda.synchronize()
+    time.sleep(1.0)
+    per_mark = max(1, int(0.005 / est_s))          # an event about every 5 ms of launches
+    marks = max(2, int(seconds / (per_mark * est_s)))
+    th = threading.Thread(target=sample, daemon=True)
+    th.start()
+    t0 = time.perf_counter()
+    events = [torch.cuda.Event(enable_timing=True)]
+    events[0].record(stream)
+    i = 0
+    for _ in range(marks):
+        for _ in range(per_mark):
+            launch(i)
+            i += 1
+        events.append(torch.cuda.Event(enable_timing=True))
+        events[-1].record(stream)
+    torch.cuda.synchronize()
+    stop.set()
+    th.join()
+    at = [events[0].elapsed_time(e) for e in events]               # ms since the first launch
+    rows, width = [], 25.0
+    for lo in np.arange(0.0, at[-1], width):
+        seg = [(at[j + 1] - at[j]) / per_mark for j in range(marks) if lo <= at[j] < lo + width]
+        smp = [x for x in samples if lo <= (x[0] - t0) * 1e3 < lo + width]
+        if seg:
+            rows.append({"ms": [float(lo), float(lo + width)], "us_per_launch": float(np.median(seg)) * 1e3,
+                         "sm_mhz": sorted({x[1] for x in smp}), "power_w_max": max([x[2] for x in smp], default=None),
+                         "reasons": sorted({hex(x[3]) for x in smp})})
+    return rows
 
 
 def main():
@@ -863,6 +946,9 @@ def main():
     ap.add_argument("--workers", type=int, default=N_WORKERS)
     ap.add_argument("--bucket", type=int, default=BUCKET)
     ap.add_argument("--launches", type=int, default=6)
+    ap.add_argument("--clock-trace", type=float, default=0.0, metavar="SECONDS",
+                    help="with --kernel: then run the launch back to back for SECONDS and report time per launch, "
+                         "SM clock and board power in rows of 25 ms")
     args = ap.parse_args()
     if args.kernel is not None:
         return run_single_kernel(args)
