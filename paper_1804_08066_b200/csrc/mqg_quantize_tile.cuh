@@ -138,7 +138,9 @@ __device__ __forceinline__ bool quantize_tile(TmaQuantizeShared<DTYPE, THREADS>&
     // SM clock at its maximum: 17.0 against 18.0 us at K = 4, 18.3 against 18.6 us at K = 6, 19.7 against
     // 20.0 us at K = 8; no difference at one and two bits, which keep the fifth CTA.  (In a long run the power
     // limit sets the clock and both forms take the same time: the instruction count decides there.)
-    constexpr bool kEarlyDraw = !NORM && !GIVEN && BITS >= 3;
+    // bf16 input (half the bytes per tile, no wait to cover) keeps the draws after the wait at every width:
+    // 32.3 / 32.1 / 32.7 / 32.4 us per 50 M elements at K = 3 / 4 / 6 / 8 against 33.2 / 32.8 / 33.6 / 32.8 us.
+    constexpr bool kEarlyDraw = !NORM && !GIVEN && DTYPE == 0 && BITS >= 3;
     uint32_t h[16];
     if (kEarlyDraw && active) draw_row_blocks_head(wv.blk0_lo + 4u * row, wv.head, c.rk, h);
     bool ok = mbar_try_wait(bar, parity);
