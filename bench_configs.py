@@ -1,7 +1,8 @@
 """The other workloads of the benchmark specification, measured after bench.py's timed region and
 reported in its JSON line under `configs`: the small launch-bound case (`configs[0]`), the layered
 AlexNet-shaped gradient with one scale per tensor (`configs[2]`) and the stress shape (`configs[4]`:
-10^9 bf16 elements, 16 workers).  The headline numbers (`value`, `roofline`) stay those of
+10^9 bf16 elements, 16 workers), and the end-to-end training loop with the host bit selector (`configs[3]`:
+the share of an iteration spent inside the library).  The headline numbers (`value`, `roofline`) stay those of
 `configs[1]`; nothing here changes them.
 
 Every kernel is timed as GROUP launches back to back between one pair of CUDA events on torch's
@@ -186,9 +187,29 @@ def stress_case(torch, mqg, lib, check, peak):
             "per_bits": rows}
 
 
+def loop_case():
+    """`configs[3]`: the whole loop (model gradients -> quantize -> fused server step -> host selector) with the
+    paper's selector; what is reported is the share of an iteration spent in the library's two calls."""
+    from paper_1804_08066_b200.train_loop import run
+    r = run(iters=40, workers=4, selector="sarsa", seed=1)
+    return {"workload": "configs[3]: 5-layer CNN (3x3 conv 32-64-128, FC 2048-256-10) on synthetic 32x32x3 images, "
+                        "batch 128 per worker, W=4, bucket 2048, host SARSA selector picks the bits from the losses; "
+                        "40 iterations",
+            "note": "the model, its autograd and the selector are the harness's; the library is the codec and the "
+                    "server step (one mqg_quantize per worker, one mqg_server_step per iteration)",
+            "parameters": r["parameters"], "libmqgrad_ms_per_iter": r["libmqgrad_ms_per_iter"],
+            "iteration_ms": r["iteration_ms"], "libmqgrad_share_pct": r["libmqgrad_share_pct"],
+            "bits_chosen_first_last": [r["bits_chosen"][0], r["bits_chosen"][-1]],
+            "first_loss": r["first_loss"], "last_loss": r["last_loss"],
+            "uplink_bytes_per_iter": r["uplink_bytes_per_iter"], "uplink_bytes_fp32": r["uplink_bytes_fp32"],
+            "paper_table3_share_pct": r["paper_table3_share_pct"]}
+
+
 def run_all(torch, mqg, lib, check, peak):
     out = {}
     for name, fn in (("config0_small", small_case), ("config2_layered", layered_case), ("config4_stress", stress_case)):
         out[name] = fn(torch, mqg, lib, check, peak)
         torch.cuda.synchronize()
+    out["config3_loop"] = loop_case()
+    torch.cuda.synchronize()
     return out
