@@ -17,6 +17,9 @@ import ctypes as C
 import numpy as np
 
 PHILOX_SEED = 2
+# executed instructions per element of quantize_tma / quantize_workers_kernel<K, bf16> (ncu, smsp__inst_executed:
+# profiles/per_width_counters_small_cases.md)
+BF16_QUANTIZE_INST_PER_ELEM = 14.3
 
 
 def _time_groups(torch, stream, launch, group, reps, warm=2):
@@ -160,6 +163,9 @@ def stress_case(torch, mqg, lib, check, peak):
     params = torch.zeros(n, dtype=torch.float32, device="cuda")
     gtab, ctab, stab = _ptrs([grad] * W), _ptrs(codes), _ptrs(scales)
     rows = []
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    sm_mhz = float(getattr(props, "clock_rate", 1965000)) / 1e3                  # the device's maximum SM clock
+    issue_peak = props.multi_processor_count * 4 * sm_mhz / 1e3                  # schedulers x GHz
     for b in range(1, 9):
         q = _time_groups(torch, stream, lambda i: check(lib.mqg_quantize_workers(
             gtab, W, n, b, B, PHILOX_SEED, ctab, stab, 1, 0, i, 0, sptr)), 2, 5, warm=1)
@@ -171,6 +177,13 @@ def stress_case(torch, mqg, lib, check, peak):
         row = {"bits": b, "quantize_all_workers": _entry(q[0], q[1], qb, peak),
                "quantize_us_per_worker": q[0] / W, "server_step": _entry(s[0], s[1], sb, peak)}
         row["quantize_all_workers"]["fp32_equivalent_grad_gbs"] = W * 4 * n / q[0] / 1e3
+        # the ceiling this kernel actually runs against: warp instructions issued per second (14.3 executed
+        # instructions per element, from the ncu counters of the bf16 instantiation) against one instruction
+        # per cycle and scheduler at the maximum SM clock
+        row["quantize_all_workers"]["issue_rate"] = {
+            "bound": "alu", "instructions_per_element": BF16_QUANTIZE_INST_PER_ELEM,
+            "achieved": W * n * BF16_QUANTIZE_INST_PER_ELEM / 32 / q[0] / 1e3, "peak": issue_peak,
+            "unit": "G warp-instructions/s", "frac": W * n * BF16_QUANTIZE_INST_PER_ELEM / 32 / q[0] / 1e3 / issue_peak}
         rows.append(row)
     timeouts = mqg.mqg_device_timeouts()
     del grad, codes, scales, params
