@@ -215,6 +215,19 @@ mqg_status mqg_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t buck
                            uint32_t step, uint64_t elem_offset, void* cuda_stream);
 
 /*
+ * The L2-norm variant for W workers' gradients of the same shape in ONE launch (the variant's
+ * counterpart of mqg_quantize_workers; related-work codec of Section 2, granularity as Section 4.1):
+ * worker w's outputs are bit-identical to mqg_quantize_l2 with worker id first_worker + w.
+ *   grads / codes / scales   HOST arrays of W DEVICE pointers, each as in mqg_quantize_l2; caller-owned
+ * Shapes the batched kernel does not take run as W launches with the same results.
+ * Errors as mqg_quantize_l2, plus MQG_ERR_TOO_MANY_WORKERS for W outside 1..MQG_MAX_WORKERS.
+ */
+mqg_status mqg_quantize_workers_l2(const void* const* grads, int W, uint64_t n, int bits, uint64_t bucket,
+                                   uint64_t seed, uint32_t* const* codes, float* const* scales,
+                                   mqg_dtype dtype, uint32_t first_worker, uint32_t step,
+                                   uint64_t elem_offset, void* cuda_stream);
+
+/*
  * The same variant with one norm per segment (per-layer scale), segment tables as in
  * mqg_quantize_segments below; the outputs go to mqg_server_step_segments.  The rows and the
  * tree of a segment start at the segment's first element.

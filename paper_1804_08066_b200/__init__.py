@@ -8,7 +8,7 @@ raises.
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_server_requantize, mqg_quantize_segments, mqg_quantize_segments_workers, mqg_server_step_segments, mqg_quantize_minmax,
-  mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_segments_l2,
+  mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_workers_l2, mqg_quantize_segments_l2,
   mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_quantize_1bit_ef, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts, mqg_check_timeouts,
   mqg_test_wait_override.
@@ -68,6 +68,7 @@ def _load() -> C.CDLL:
         "mqg_quantize_segments_workers": (i32, [vp, i32, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_quantize_1bit_ef": (i32, [vp, vp, u64, u64, vp, vp, i32, vp]),
         "mqg_quantize_l2": (i32, [vp, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
+        "mqg_quantize_workers_l2": (i32, [vp, i32, u64, i32, u64, u64, vp, vp, i32, u32, u32, u64, vp]),
         "mqg_l2_workspace_floats": (C.c_size_t, [i32, vp]),
         "mqg_quantize_segments_l2": (i32, [vp, i32, vp, vp, i32, u64, vp, vp, i32, u32, u32, u64, vp,
                                            C.c_size_t, vp]),
@@ -196,6 +197,20 @@ def mqg_quantize_workers(grads, W: int, n: int, bits: int, bucket: int, seed: in
                                      seed & 0xFFFFFFFFFFFFFFFF, _ptr_table(codes, "codes"),
                                      _ptr_table(scales, "scales"), dtypes.pop(), first_worker, step,
                                      elem_offset, _stream()))
+
+
+def mqg_quantize_workers_l2(grads, W: int, n: int, bits: int, bucket: int, seed: int, codes, scales,
+                            first_worker: int = 0, step: int = 0, elem_offset: int = 0) -> None:
+    """The L2-norm scale variant for W workers' gradients (lists of W tensors) in one launch."""
+    if len(grads) != W or len(codes) != W or len(scales) != W:
+        raise ValueError("grads, codes and scales must each hold W tensors")
+    dtypes = {_grad_dtype(g) for g in grads}
+    if len(dtypes) != 1:
+        raise TypeError("all gradients must have the same dtype")
+    _check(_lib.mqg_quantize_workers_l2(_ptr_table(grads, "grads"), W, n, bits, bucket,
+                                        seed & 0xFFFFFFFFFFFFFFFF, _ptr_table(codes, "codes"),
+                                        _ptr_table(scales, "scales"), dtypes.pop(), first_worker, step,
+                                        elem_offset, _stream()))
 
 
 def mqg_dequant_accumulate(codes, scales, W: int, bits: int, n: int, acc, bucket: int,

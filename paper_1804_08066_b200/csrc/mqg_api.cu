@@ -217,7 +217,7 @@ mqg_status mqg_quantize_workers(const void* const* grads, int W, uint64_t n, int
     if (mqg::quantize_workers_applies(W, n, bucket, elem_offset)) {
         const cudaError_t err = mqg::launch_quantize_workers(grads, W, n, bits, bucket, seed, codes, scales,
                                                              (int)dtype, first_worker, step, elem_offset,
-                                                             stream);
+                                                             false, stream);
         if (err != cudaSuccess) return cuda_fail("mqg_quantize_workers", err);
         return MQG_OK;
     }
@@ -516,6 +516,45 @@ mqg_status mqg_quantize_l2(const void* grad, uint64_t n, int bits, uint64_t buck
                                                     worker, step, elem_offset,
                                                     static_cast<cudaStream_t>(cuda_stream));
     if (err != cudaSuccess) return cuda_fail("mqg_quantize_l2", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_quantize_workers_l2(const void* const* grads, int W, uint64_t n, int bits, uint64_t bucket,
+                                   uint64_t seed, uint32_t* const* codes, float* const* scales,
+                                   mqg_dtype dtype, uint32_t first_worker, uint32_t step,
+                                   uint64_t elem_offset, void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (W < 1 || W > MQG_MAX_WORKERS)
+        return fail(MQG_ERR_TOO_MANY_WORKERS, "W = %d outside 1..%d", W, MQG_MAX_WORKERS);
+    if (n == 0) return MQG_OK;
+    if ((bucket < n ? bucket : n) > (uint64_t)mqg::kMaxFusedBucket)
+        return fail(MQG_ERR_INVALID, "mqg_quantize_workers_l2 supports buckets of at most %d elements; use "
+                    "mqg_quantize_segments_l2 for longer ones", mqg::kMaxFusedBucket);
+    if (!grads || !codes || !scales) return fail(MQG_ERR_INVALID, "grads, codes or scales is null");
+    for (int w = 0; w < W; ++w) {
+        if (!grads[w] || !codes[w] || !scales[w])
+            return fail(MQG_ERR_INVALID, "worker %d: grad, codes or scales is null", w);
+        if (!aligned16(grads[w])) return fail(MQG_ERR_ALIGN, "worker %d: grad not 16-byte aligned", w);
+        if (!aligned16(codes[w])) return fail(MQG_ERR_ALIGN, "worker %d: codes not 16-byte aligned", w);
+        if (!aligned4(scales[w])) return fail(MQG_ERR_ALIGN, "worker %d: scales not 4-byte aligned", w);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (mqg::quantize_workers_applies(W, n, bucket, elem_offset)) {
+        const cudaError_t err = mqg::launch_quantize_workers(grads, W, n, bits, bucket, seed, codes, scales,
+                                                             (int)dtype, first_worker, step, elem_offset,
+                                                             true, stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_quantize_workers_l2", err);
+        return MQG_OK;
+    }
+    // shapes the batched kernel does not take: one launch per worker, same results
+    for (int w = 0; w < W; ++w) {
+        const mqg_status st = mqg_quantize_l2(grads[w], n, bits, bucket, seed, codes[w], scales[w], dtype,
+                                              first_worker + (uint32_t)w, step, elem_offset, cuda_stream);
+        if (st != MQG_OK) return st;
+    }
     return MQG_OK;
 }
 

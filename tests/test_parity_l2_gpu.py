@@ -236,3 +236,45 @@ def test_alexnet_shaped_layers_one_norm_per_tensor():
         words = O.pack(q, bits)
         full = (m * bits) // 32
         assert np.array_equal(got[int(coff[j]):int(coff[j]) + full], words[:full]), j
+
+
+def assert_workers_parity(xs, bits, bucket, bf16=False, seed=0, first_worker=0, step=0, elem_offset=0):
+    """mqg_quantize_workers_l2 (one launch for all workers) against the CPU checker, worker by worker."""
+    W, n = len(xs), xs[0].size
+    gs = [to_dev(x.view(np.int16)).view(torch.bfloat16) if bf16 else to_dev(x) for x in xs]
+    codes = [Guarded(mqg.mqg_code_words(n, bits), torch.int32) for _ in range(W)]
+    scales = [Guarded(mqg.mqg_num_buckets(n, bucket), torch.float32) for _ in range(W)]
+    mqg.mqg_quantize_workers_l2(gs, W, n, bits, bucket, seed, [c.view for c in codes], [s.view for s in scales],
+                                first_worker=first_worker, step=step, elem_offset=elem_offset)
+    torch.cuda.synchronize()
+    for w in range(W):
+        codes[w].check_guards(), scales[w].check_guards()
+        c_ref, s_ref = O.quantize_l2(xs[w], bits, bucket, seed, worker=first_worker + w, step=step,
+                                     elem_offset=elem_offset, dtype="bf16" if bf16 else "f32")
+        assert bits_equal(scales[w].numpy(np.float32), s_ref) == 0, "worker %d: scales differ" % w
+        assert np.array_equal(codes[w].numpy(np.uint32), c_ref), "worker %d: codes differ" % w
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_workers_in_one_launch(bits):
+    """Four workers, bucket 2048 (two warps per bucket), ragged last tile and row."""
+    n = 5 * 4096 * 9 + 2048 + 21
+    xs = [wl.laplace(n, 1e-4, config=2, worker=w) for w in range(4)]
+    assert_workers_parity(xs, bits, 2048, seed=7, first_worker=3, step=bits)
+
+
+@pytest.mark.parametrize("bits", [1, 4, 7])
+@pytest.mark.parametrize("n,bucket", [
+    (300_000 + 9, 4096), (70_000, 512), (40_000, 96),       # four warps; 16-row shuffles; a shape of W launches
+    (1 << 20, 1024), (33, 32),
+])
+def test_workers_shapes(bits, n, bucket):
+    xs = [wl.normal(n, 1e-3, config=1, worker=10 + w) for w in range(3)]
+    assert_workers_parity(xs, bits, bucket, seed=n, step=2)
+
+
+@pytest.mark.parametrize("bits", [2, 5, 8])
+def test_workers_bf16_and_offset_draws(bits):
+    n = 3 * 4096 * 11 + 4096
+    xs = [wl.student_t_bf16(n, config=5, worker=w) for w in range(2)]
+    assert_workers_parity(xs, bits, 4096, bf16=True, seed=5, first_worker=1, elem_offset=8 * 12345)
