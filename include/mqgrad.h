@@ -158,6 +158,18 @@ mqg_status mqg_server_requantize(const uint32_t* const* codes, const float* cons
  */
 mqg_status mqg_quantize_minmax(const void* grad, uint64_t n, int bits, uint64_t bucket, uint32_t* codes,
                                float* ranges, mqg_dtype dtype, void* cuda_stream);
+/*
+ * The (min, max) variant for W workers' gradients of the same shape in ONE launch (the variant's
+ * counterpart of mqg_quantize_workers; the scheme the footnote of Section 3.2 points to): worker w's
+ * outputs are bit-identical to mqg_quantize_minmax on its gradient.
+ *   grads / codes / ranges   HOST arrays of W DEVICE pointers, each as in mqg_quantize_minmax; caller-owned
+ * Shapes the batched kernel does not take run as W calls with the same results.
+ * Errors as mqg_quantize_minmax, plus MQG_ERR_TOO_MANY_WORKERS for W outside 1..MQG_MAX_WORKERS.
+ */
+mqg_status mqg_quantize_workers_minmax(const void* const* grads, int W, uint64_t n, int bits, uint64_t bucket,
+                                       uint32_t* const* codes, float* const* ranges, mqg_dtype dtype,
+                                       void* cuda_stream);
+
 
 /*
  * Server side of the variant: mqg_dequant_accumulate and mqg_server_step with x^ as above and the

@@ -8,6 +8,7 @@ raises.
 Function names and argument order follow the C ABI:
   mqg_quantize, mqg_quantize_workers, mqg_dequant_accumulate, mqg_apply, mqg_server_step,
   mqg_server_requantize, mqg_quantize_segments, mqg_quantize_segments_workers, mqg_server_step_segments, mqg_quantize_minmax,
+  mqg_quantize_workers_minmax,
   mqg_dequant_accumulate_minmax, mqg_server_step_minmax, mqg_quantize_l2, mqg_quantize_workers_l2, mqg_quantize_segments_l2,
   mqg_l2_workspace_floats, mqg_quantize_segments_l2_static, mqg_quantize_1bit_ef, mqg_code_words, mqg_num_buckets,
   mqg_wire_bytes, mqg_last_error, mqg_version, mqg_device_timeouts, mqg_check_timeouts,
@@ -59,6 +60,7 @@ def _load() -> C.CDLL:
         "mqg_dequant_accumulate": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
         "mqg_apply": (i32, [vp, vp, f32, u64, vp]),
         "mqg_quantize_minmax": (i32, [vp, u64, i32, u64, vp, vp, i32, vp]),
+        "mqg_quantize_workers_minmax": (i32, [vp, i32, u64, i32, u64, vp, vp, i32, vp]),
         "mqg_dequant_accumulate_minmax": (i32, [vp, vp, i32, i32, u64, vp, u64, i32, vp]),
         "mqg_server_step_minmax": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
         "mqg_server_step": (i32, [vp, vp, i32, i32, u64, u64, vp, f32, vp, vp]),
@@ -231,6 +233,18 @@ def mqg_server_step(codes, scales, W: int, bits: int, n: int, bucket: int, param
                                 n, bucket, _dev_ptr(params, "params") if n else None, lr,
                                 _dev_ptr(acc_out, "acc_out") if acc_out is not None else None,
                                 _stream()))
+
+
+def mqg_quantize_workers_minmax(grads, W: int, n: int, bits: int, bucket: int, codes, ranges) -> None:
+    """The (min, max) variant for W workers' gradients (lists of W tensors) in one launch."""
+    if len(grads) != W or len(codes) != W or len(ranges) != W:
+        raise ValueError("grads, codes and ranges must each hold W tensors")
+    dtypes = {_grad_dtype(g) for g in grads}
+    if len(dtypes) != 1:
+        raise TypeError("all gradients must have the same dtype")
+    _check(_lib.mqg_quantize_workers_minmax(_ptr_table(grads, "grads"), W, n, bits, bucket,
+                                            _ptr_table(codes, "codes"), _ptr_table(ranges, "ranges"),
+                                            dtypes.pop(), _stream()))
 
 
 def mqg_quantize_minmax(grad, n: int, bits: int, bucket: int, codes, ranges) -> None:

@@ -217,7 +217,7 @@ mqg_status mqg_quantize_workers(const void* const* grads, int W, uint64_t n, int
     if (mqg::quantize_workers_applies(W, n, bucket, elem_offset)) {
         const cudaError_t err = mqg::launch_quantize_workers(grads, W, n, bits, bucket, seed, codes, scales,
                                                              (int)dtype, first_worker, step, elem_offset,
-                                                             false, stream);
+                                                             0, stream);
         if (err != cudaSuccess) return cuda_fail("mqg_quantize_workers", err);
         return MQG_OK;
     }
@@ -246,6 +246,39 @@ mqg_status mqg_quantize_minmax(const void* grad, uint64_t n, int bits, uint64_t 
         ? mqg::launch_quantize_range_fused(grad, n, bits, bucket, codes, ranges, (int)dtype, stream)
         : mqg::launch_quantize_range_general(grad, n, bits, bucket, codes, ranges, (int)dtype, stream);
     if (err != cudaSuccess) return cuda_fail("mqg_quantize_minmax", err);
+    return MQG_OK;
+}
+
+mqg_status mqg_quantize_workers_minmax(const void* const* grads, int W, uint64_t n, int bits, uint64_t bucket,
+                                       uint32_t* const* codes, float* const* ranges, mqg_dtype dtype,
+                                       void* cuda_stream)
+{
+    if (mqg_status st = check_bits(bits)) return st;
+    if (mqg_status st = check_bucket(n, bucket)) return st;
+    if (dtype != MQG_F32 && dtype != MQG_BF16) return fail(MQG_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (W < 1 || W > MQG_MAX_WORKERS)
+        return fail(MQG_ERR_TOO_MANY_WORKERS, "W = %d outside 1..%d", W, MQG_MAX_WORKERS);
+    if (n == 0) return MQG_OK;
+    if (!grads || !codes || !ranges) return fail(MQG_ERR_INVALID, "grads, codes or ranges is null");
+    for (int w = 0; w < W; ++w) {
+        if (!grads[w] || !codes[w] || !ranges[w])
+            return fail(MQG_ERR_INVALID, "worker %d: grad, codes or ranges is null", w);
+        if (!aligned16(grads[w])) return fail(MQG_ERR_ALIGN, "worker %d: grad not 16-byte aligned", w);
+        if (!aligned16(codes[w])) return fail(MQG_ERR_ALIGN, "worker %d: codes not 16-byte aligned", w);
+        if (!aligned8(ranges[w])) return fail(MQG_ERR_ALIGN, "worker %d: ranges not 8-byte aligned", w);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (mqg::quantize_workers_applies(W, n, bucket, 0)) {
+        const cudaError_t err = mqg::launch_quantize_workers(grads, W, n, bits, bucket, 0, codes, ranges,
+                                                             (int)dtype, 0, 0, 0, 1, stream);
+        if (err != cudaSuccess) return cuda_fail("mqg_quantize_workers_minmax", err);
+        return MQG_OK;
+    }
+    // shapes the batched kernel does not take: one call per worker, same results
+    for (int w = 0; w < W; ++w) {
+        const mqg_status st = mqg_quantize_minmax(grads[w], n, bits, bucket, codes[w], ranges[w], dtype, cuda_stream);
+        if (st != MQG_OK) return st;
+    }
     return MQG_OK;
 }
 
@@ -545,7 +578,7 @@ mqg_status mqg_quantize_workers_l2(const void* const* grads, int W, uint64_t n, 
     if (mqg::quantize_workers_applies(W, n, bucket, elem_offset)) {
         const cudaError_t err = mqg::launch_quantize_workers(grads, W, n, bits, bucket, seed, codes, scales,
                                                              (int)dtype, first_worker, step, elem_offset,
-                                                             true, stream);
+                                                             2, stream);
         if (err != cudaSuccess) return cuda_fail("mqg_quantize_workers_l2", err);
         return MQG_OK;
     }

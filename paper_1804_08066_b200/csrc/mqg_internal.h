@@ -40,12 +40,13 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
 
 // One launch for W >= 2 workers' gradients of the same shape (host arrays of device pointers);
 // worker w draws as worker id first_worker + w.  Only when quantize_workers_applies() holds.
-// l2_norm: the L2-norm scale variant's tile code instead of the max-abs one.
+// mode: 0 = the main codec, 1 = the (min, max) variant (`scales[w]` then points at worker w's ranges, two floats
+// per bucket; seed, first_worker, step and elem_offset are not used), 2 = the L2-norm scale variant.
 bool quantize_workers_applies(int W, uint64_t n, uint64_t bucket, uint64_t elem_offset);
 cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n, int bits,
                                     uint64_t bucket, uint64_t seed, uint32_t* const* codes,
                                     float* const* scales, int dtype, uint32_t first_worker,
-                                    uint32_t step, uint64_t elem_offset, bool l2_norm, cudaStream_t stream);
+                                    uint32_t step, uint64_t elem_offset, int mode, cudaStream_t stream);
 
 // (min, max) nearest-rounding variant.  ranges[2b] = lo, ranges[2b + 1] = hi of bucket b.
 // Fused one-pass kernel for buckets of at most 4096 elements; otherwise the general launches

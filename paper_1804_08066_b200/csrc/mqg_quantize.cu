@@ -284,7 +284,7 @@ struct WorkerTable {
     PhiloxHead head[kMaxWorkers];
 };
 
-template <int BITS, int DTYPE, bool SHUFFLE, bool NORM>
+template <int BITS, int DTYPE, bool SHUFFLE, int MODE>
 __global__ void __launch_bounds__(128, 4)
 quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_constant__ QuantizeArgs a,
                         const __grid_constant__ TmaQuantizeConsts c, uint32_t total_tiles,
@@ -302,7 +302,10 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
         for (int s = 0; s < kQuantStages; ++s) mbar_init(smem_u32(&sh.bar[s]), 1);
         fence_barrier_init();
     }
-    if (t < 3 * (THREADS / 32)) (&sh.slots[0][0])[t] = 0u;
+    if (t < 3 * (THREADS / 32)) {
+        (&sh.slots[0][0])[t] = 0u;     // = kOrderedMaxIdentity
+        (&sh.slots_lo[0][0])[t] = kOrderedMinIdentity;
+    }
     grid_dependency_release();
     __syncthreads();
     grid_dependency_wait();            // nothing above touches global memory
@@ -346,12 +349,22 @@ quantize_workers_kernel(const __grid_constant__ WorkerTable tab, const __grid_co
             auto refill = [&](uint32_t stage, uint32_t bar) {
                 if (vfill < total_tiles) load_tile(fill, stage, bar);
             };
-            if (tile < c.full_tiles)
-                ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM>(sh, wv, a, c, k, rot, tile, refill,
-                                                                               local_bucket, scale_writer);
-            else
-                ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM>(sh, wv, a, c, k, rot, tile, refill,
-                                                                                local_bucket, scale_writer);
+            if constexpr (MODE == kRange) {
+                if (tile < c.full_tiles)
+                    ok = range_quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE>(sh, wv, a, k, rot, tile, refill,
+                                                                                   local_bucket, scale_writer);
+                else
+                    ok = range_quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE>(sh, wv, a, k, rot, tile, refill,
+                                                                                    local_bucket, scale_writer);
+            } else {
+                constexpr bool NORM = MODE == kNorm;
+                if (tile < c.full_tiles)
+                    ok = quantize_tile<BITS, DTYPE, THREADS, true, SHUFFLE, NORM>(sh, wv, a, c, k, rot, tile, refill,
+                                                                                   local_bucket, scale_writer);
+                else
+                    ok = quantize_tile<BITS, DTYPE, THREADS, false, SHUFFLE, NORM>(sh, wv, a, c, k, rot, tile, refill,
+                                                                                    local_bucket, scale_writer);
+            }
             vfill += stride;
             if (vfill < total_tiles) advance(fill, stride);
         }
@@ -541,12 +554,12 @@ cudaError_t launch_quantize_fused(const void* grad, uint64_t n, int bits, uint64
     return cudaErrorInvalidValue;
 }
 
-template <int BITS, int DTYPE, bool SHUFFLE, bool NORM>
+template <int BITS, int DTYPE, bool SHUFFLE, int MODE>
 static cudaError_t launch_workers_inst(const WorkerTable& tab, const QuantizeArgs& a,
                                        const TmaQuantizeConsts& c, uint32_t total_tiles,
                                        unsigned int* timeouts, cudaStream_t stream)
 {
-    auto kernel = quantize_workers_kernel<BITS, DTYPE, SHUFFLE, NORM>;
+    auto kernel = quantize_workers_kernel<BITS, DTYPE, SHUFFLE, MODE>;
     static std::atomic<int> grid_cap[64];                  // per device; 0 = not yet queried (zero-initialised)
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -567,16 +580,16 @@ static cudaError_t launch_workers_inst(const WorkerTable& tab, const QuantizeArg
     return launch_pdl(kernel, grid, 128, stream, tab, a, c, total_tiles, timeouts);
 }
 
-template <int BITS, bool NORM>
+template <int BITS, int MODE>
 static cudaError_t launch_workers_bits(const WorkerTable& tab, const QuantizeArgs& a,
                                        const TmaQuantizeConsts& c, uint32_t total_tiles, int dtype,
                                        bool shuffle, unsigned int* timeouts, cudaStream_t stream)
 {
     if (dtype == 0)
-        return shuffle ? launch_workers_inst<BITS, 0, true, NORM>(tab, a, c, total_tiles, timeouts, stream)
-                       : launch_workers_inst<BITS, 0, false, NORM>(tab, a, c, total_tiles, timeouts, stream);
-    return shuffle ? launch_workers_inst<BITS, 1, true, NORM>(tab, a, c, total_tiles, timeouts, stream)
-                   : launch_workers_inst<BITS, 1, false, NORM>(tab, a, c, total_tiles, timeouts, stream);
+        return shuffle ? launch_workers_inst<BITS, 0, true, MODE>(tab, a, c, total_tiles, timeouts, stream)
+                       : launch_workers_inst<BITS, 0, false, MODE>(tab, a, c, total_tiles, timeouts, stream);
+    return shuffle ? launch_workers_inst<BITS, 1, true, MODE>(tab, a, c, total_tiles, timeouts, stream)
+                   : launch_workers_inst<BITS, 1, false, MODE>(tab, a, c, total_tiles, timeouts, stream);
 }
 
 bool quantize_workers_applies(int W, uint64_t n, uint64_t bucket, uint64_t elem_offset)
@@ -594,7 +607,7 @@ bool quantize_workers_applies(int W, uint64_t n, uint64_t bucket, uint64_t elem_
 cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n, int bits,
                                     uint64_t bucket, uint64_t seed, uint32_t* const* codes,
                                     float* const* scales, int dtype, uint32_t first_worker,
-                                    uint32_t step, uint64_t elem_offset, bool l2_norm, cudaStream_t stream)
+                                    uint32_t step, uint64_t elem_offset, int mode, cudaStream_t stream)
 {
     QuantizeArgs a;
     const uint64_t rpb = fill_args(a, grads[0], n, bits, bucket, seed, codes[0], scales[0], first_worker,
@@ -616,8 +629,9 @@ cudaError_t launch_quantize_workers(const void* const* grads, int W, uint64_t n,
     const bool shuffle = rpb <= 32;
     switch (bits) {
 #define MQG_WORKERS_CASE(B) \
-        case B: return l2_norm ? launch_workers_bits<B, true>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream) \
-                               : launch_workers_bits<B, false>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream)
+        case B: return mode == kNorm ? launch_workers_bits<B, kNorm>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream) \
+                     : mode == kRange ? launch_workers_bits<B, kRange>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream) \
+                     : launch_workers_bits<B, kMaxAbs>(tab, a, c, total_tiles, dtype, shuffle, timeouts, stream)
         MQG_WORKERS_CASE(1); MQG_WORKERS_CASE(2); MQG_WORKERS_CASE(3); MQG_WORKERS_CASE(4);
         MQG_WORKERS_CASE(5); MQG_WORKERS_CASE(6); MQG_WORKERS_CASE(7); MQG_WORKERS_CASE(8);
 #undef MQG_WORKERS_CASE

@@ -170,3 +170,44 @@ def test_argument_errors_and_empty_input():
     assert e.value.status == mqg.MQG_ERR_ALIGN
     mqg.mqg_quantize_minmax(g, 0, 4, 512, c, r)
     mqg.mqg_server_step_minmax([c], [r], 1, 4, 0, 512, g, 0.1)
+
+
+def assert_workers_parity(xs, bits, bucket, bf16=False):
+    """mqg_quantize_workers_minmax (one launch for all workers) against the CPU checker, worker by worker."""
+    W, n = len(xs), xs[0].size
+    gs = [to_dev(x.view(np.int16)).view(torch.bfloat16) if bf16 else to_dev(x) for x in xs]
+    codes = [Guarded(mqg.mqg_code_words(n, bits), torch.int32) for _ in range(W)]
+    ranges = [Guarded(2 * mqg.mqg_num_buckets(n, bucket), torch.float32) for _ in range(W)]
+    mqg.mqg_quantize_workers_minmax(gs, W, n, bits, bucket, [c.view for c in codes], [r.view for r in ranges])
+    torch.cuda.synchronize()
+    for w in range(W):
+        codes[w].check_guards(), ranges[w].check_guards()
+        c_ref, r_ref = O.quantize_minmax(xs[w], bits, bucket, dtype="bf16" if bf16 else "f32")
+        assert bits_equal(ranges[w].numpy(np.float32), r_ref) == 0, "worker %d: ranges differ" % w
+        assert np.array_equal(codes[w].numpy(np.uint32), c_ref), "worker %d: codes differ" % w
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_workers_in_one_launch(bits):
+    """Four workers, bucket 2048, ragged last tile and ragged last row (its padding must not widen a range)."""
+    n = 5 * 4096 * 9 + 2048 + 21
+    xs = [wl.laplace(n, 1e-4, config=2, worker=w) + np.float32(1e-4 * w) for w in range(4)]
+    assert_workers_parity(xs, bits, 2048)
+
+
+@pytest.mark.parametrize("bits", [1, 4, 7])
+@pytest.mark.parametrize("n,bucket", [
+    (300_000 + 9, 4096), (70_000, 512), (40_000, 96),       # four warps; 16-row shuffles; a shape of W calls
+    (1 << 20, 1024), (33, 32),
+])
+def test_workers_shapes(bits, n, bucket):
+    xs = [wl.normal(n, 1e-3, config=1, worker=10 + w) for w in range(3)]
+    xs[1][: min(n, bucket)] = np.float32(0.25)              # a constant bucket: every code 0
+    assert_workers_parity(xs, bits, bucket)
+
+
+@pytest.mark.parametrize("bits", [2, 5, 8])
+def test_workers_bf16(bits):
+    n = 3 * 4096 * 11 + 4096
+    xs = [wl.student_t_bf16(n, config=5, worker=w) for w in range(2)]
+    assert_workers_parity(xs, bits, 4096, bf16=True)
